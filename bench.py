@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the ASL prefill hot path (score -> pool -> rank statistic ->
+per-head top-k -> K/V compaction) on synthetic long-context tensors.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+
+One "step" = one pass of the whole path over one layer's tensors of the
+workload.  Prints ONE JSON line.  Inputs are seeded synthetic tensors shaped
+like the 128K-token single-request workload (32 q heads / 8 kv heads, d=128,
+w=64, budget 4096); several layers' tensors stay resident and the steps rotate
+through them, so every step streams a K larger than L2 that it has not touched
+for at least two steps.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_07667_b200 import inputs as I   # noqa: E402
+
+METRIC = "obs-window score+select+compact: context tokens/s/layer"
+UNIT = "tokens/s/layer"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def algorithmic_work(wl):
+    """Algorithmic bytes and flops of one layer's pass: K read once, Q once, only
+    kept K/V rows gathered (read + write), score vectors written and re-read by
+    the pooling, ranking and selection stages, one QK^T."""
+    d, Hk, Hq, w = wl.head_dim, wl.n_kv_heads, wl.n_q_heads, wl.window
+    n_tot = wl.total_tokens
+    T_tot = n_tot - wl.batch * w
+    kept = sum(wl.kept(b) for b in range(wl.batch))
+    k_bytes = n_tot * Hk * d * 2
+    q_bytes = wl.batch * w * Hq * d * 2
+    gather = 4 * kept * Hk * d * 2
+    score = 3 * (Hk + 1) * T_tot * 4 + kept * Hk * 4
+    flops = 2.0 * w * d * n_tot * Hq
+    return {"bytes": k_bytes + q_bytes + gather + score, "k_bytes": k_bytes, "flops": flops,
+            "exps": float(w) * Hq * n_tot}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        mhz, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                mhz.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(mhz), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------------------------
+def oracle_step(wl, x, layer, controllers, heads=None):
+    """One layer of the path by the fp64 oracle (optionally only the first `heads` kv heads)."""
+    from oracle import asl_oracle as O
+    cu = wl.cu_seqlens()
+    Hk = wl.n_kv_heads if heads is None else heads
+    for b in range(wl.batch):
+        n, w = wl.seqlens[b], wl.window
+        q = O.widen_bf16(x["q_obs"][b][: Hk * wl.group])
+        k = O.widen_bf16(x["k"][cu[b]:cu[b + 1], :Hk])
+        P, agg = O.score_layer(q, k, wl.group, wl.pool_kernel, wl.pool_mode)
+        controllers[b].step(layer, agg)
+        kk = O.kept_count(wl.budgets[b], n, w)
+        for h in range(Hk):
+            idx = O.select_topk(P[h], kk, n, w)
+            O.compact_rows(x["k"][cu[b]:cu[b + 1]], idx, h)
+            O.compact_rows(x["v"][cu[b]:cu[b + 1]], idx, h)
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(wl, layer_sets, steps, warmup, heads):
+    from oracle import asl_oracle as O
+    ctl = [O.SelectionController(wl.budgets[b], wl.window, wl.l_min, wl.l_obs, wl.tau) for b in range(wl.batch)]
+    for i in range(warmup):
+        oracle_step(wl, layer_sets[i % len(layer_sets)], i, ctl, heads)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        oracle_step(wl, layer_sets[i % len(layer_sets)], warmup + i, ctl, heads)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    frac = heads / wl.n_kv_heads
+    return wl.total_tokens * frac / dt, dt
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    wl = I.workload(args.workload, seed=args.seed)
+    heads = 1
+    sets = [I.layer_inputs(wl, l, args.seed) for l in range(2)]
+    np.dot(np.ones((64, 64)), np.ones((64, 64)))
+    value, dt = time_oracle(wl, sets, args.steps, args.warmup, heads)
+    cores = oracle_threads()
+    sample = (f"each step: the whole path of one layer for kv head 0 and its {wl.group} query heads "
+              f"(1/{wl.n_kv_heads} of the scoring, top-k and compaction; the rank statistic in full), "
+              f"value scaled by that fraction")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "seqlens": list(wl.seqlens), "window": wl.window,
+                       "budgets": list(wl.budgets), "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv", "d": wl.head_dim},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_07667_b200 import binding as B
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = I.workload(args.workload, seed=args.seed)
+    work = algorithmic_work(wl)
+    pk = peaks()
+
+    # resident inputs: a few layers' tensors, rotated (each rank draws its own seed: independent requests)
+    n_sets = args.layer_sets
+    host_sets = [I.layer_inputs(wl, l, args.seed + rank) for l in range(n_sets)]
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    host_pinned = [{k: pin(x[k]) for k in ("q_obs", "k", "v")} for x in host_sets]
+    dev_sets = [{k: t.cuda(non_blocking=True).view(torch.bfloat16) for k, t in hp.items()} for hp in host_pinned]
+    torch.cuda.synchronize()
+
+    path = B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
+                       pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
+                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(i, marks=None):
+        s = dev_sets[i % n_sets]
+        if marks is None:
+            path.run_layer(s["q_obs"], s["k"], s["v"], i)
+            return
+        # same calls as run_layer, with events between the stages (stage timing run only)
+        ctx, ws, wsb = path.ctx, path.workspace, path.ws_bytes
+        rows = path.n_rows(i)
+        e = [ev() for _ in range(5)]
+        e[0].record(stream)
+        B.asl_score_layer(ctx, s["q_obs"], s["k"], path.scores_kv, path.scores_agg, ws, wsb)
+        e[1].record(stream)
+        B.asl_rank_stat(ctx, path.scores_agg, i, rows, path.rank_ring, path.stat, ws, wsb)
+        e[2].record(stream)
+        B.asl_select_topk(ctx, path.scores_kv, wl.n_kv_heads, path.idx, ws, wsb)
+        e[3].record(stream)
+        B.asl_compact_kv(ctx, s["k"], s["v"], path.idx, path.k_out, path.v_out)
+        e[4].record(stream)
+        marks.append(e)
+
+    # ---- warm-up, then the timed region: EXACTLY `steps` steps ----
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = B.asl_launch_count(path.ctx)
+    score_marks = []
+    t_start, t_end = ev(), ev()
+    barrier()
+    t_start.record(stream)
+    for i in range(args.steps):
+        s = dev_sets[(args.warmup + i) % n_sets]
+        a, b_ = ev(), ev()
+        a.record(stream)
+        B.asl_score_layer(path.ctx, s["q_obs"], s["k"], path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
+        b_.record(stream)
+        score_marks.append((a, b_))
+        li = args.warmup + i
+        rows = path.n_rows(li)
+        path._fork.record(stream)
+        path.side.wait_event(path._fork)
+        B.asl_rank_stat(path.ctx, path.scores_agg, li, rows, path.rank_ring, path.stat, path.workspace, path.ws_bytes,
+                        path.side)
+        path._join.record(path.side)
+        B.asl_select_topk(path.ctx, path.scores_kv, wl.n_kv_heads, path.idx, path.workspace, path.ws_bytes)
+        B.asl_compact_kv(path.ctx, s["k"], s["v"], path.idx, path.k_out, path.v_out)
+        stream.wait_event(path._join)
+    t_end.record(stream)
+    barrier()
+    launches = B.asl_launch_count(path.ctx) - launches0
+    time.sleep(0.2)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t_start.elapsed_time(t_end)
+    score_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in score_marks]))
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * wl.total_tokens / (ms_step * 1e-3)
+
+    # ---- per-stage times (serialised, outside the timed region) ----
+    marks = []
+    for i in range(min(args.steps, 8)):
+        step(args.warmup + args.steps + i, marks)
+    torch.cuda.synchronize()
+    stage_ms = [float(np.mean([m[j].elapsed_time(m[j + 1]) for m in marks])) for j in range(4)]
+
+    # ---- end to end through the C ABI with host buffers ----
+    e2e_steps = max(2, min(args.steps, args.e2e_steps))
+    q_d, k_d, v_d = (torch.empty_like(dev_sets[0][k]) for k in ("q_obs", "k", "v"))
+    idx_h = torch.empty(path.idx.shape, dtype=torch.int32).pin_memory()
+    ko_h = torch.empty(path.k_out.shape, dtype=torch.bfloat16).pin_memory()
+    vo_h = torch.empty(path.v_out.shape, dtype=torch.bfloat16).pin_memory()
+    st_h = torch.empty(path.stat.shape, dtype=torch.uint8).pin_memory()
+
+    def e2e_step(i):
+        hp = host_pinned[i % n_sets]
+        q_d.view(torch.int16).copy_(hp["q_obs"], non_blocking=True)
+        k_d.view(torch.int16).copy_(hp["k"], non_blocking=True)
+        v_d.view(torch.int16).copy_(hp["v"], non_blocking=True)
+        path.run_layer(q_d, k_d, v_d, i)
+        idx_h.copy_(path.idx, non_blocking=True)
+        ko_h.copy_(path.k_out, non_blocking=True)
+        vo_h.copy_(path.v_out, non_blocking=True)
+        st_h.copy_(path.stat, non_blocking=True)
+
+    path.reset()
+    e2e_step(0)
+    barrier()
+    e0, e1 = ev(), ev()
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(1 + i)
+    e1.record(stream)
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / e2e_steps
+    h2d = sum(host_pinned[0][k].numel() * 2 for k in ("q_obs", "k", "v"))
+    d2h = idx_h.numel() * 4 + ko_h.numel() * 2 + vo_h.numel() * 2 + st_h.numel()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the whole step and of the scorer ----
+    hbm = pk["hbm_gbs"]
+    tf = pk["bf16_tflops"]
+    t_hbm = work["bytes"] / (hbm * 1e9)
+    t_mma = work["flops"] / (tf * 1e12)
+    bound = "hbm" if t_hbm >= t_mma else "tensor"
+    if bound == "hbm":
+        achieved = work["k_bytes"] / (score_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm}
+    else:
+        achieved = work["flops"] / (score_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": tf, "unit": "TFLOP/s", "frac": achieved / tf}
+    roof.update({"traffic": None, "kernel": "asl_score_layer (scorer passes + pooling)", "kernel_ms": score_ms,
+                 "peak_source": pk["source"], "step_roofline_us": max(t_hbm, t_mma) * 1e6,
+                 "step_frac": max(t_hbm, t_mma) / (ms_step * 1e-3)})
+
+    # ---- the oracle on the host cores, bounded sample ----
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, dt = time_oracle(wl, host_sets, 2, 1, 1)
+        cpu = {"value": v, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+               "sample": f"2 layers, kv head 0 with its {wl.group} query heads (1/{wl.n_kv_heads} of scoring, top-k and "
+                         f"compaction, rank statistic in full), scaled by that fraction; {dt:.2f} s per sampled layer"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "seqlens": list(wl.seqlens), "window": wl.window,
+                       "budgets": list(wl.budgets), "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv", "d": wl.head_dim,
+                       "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"],
+                       "l2": f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
+                             f"{work['k_bytes'] / 1e6:.0f} MB per layer",
+                       "parallelism": f"replicas x{world}"},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": world * wl.total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": int(launches), "clocks": clocks,
+            "stages_ms": {"score+pool": stage_ms[0], "rank_stat": stage_ms[1], "topk": stage_ms[2],
+                          "compact": stage_ms[3]}}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--layer-sets", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,162 @@
+/* asl.h -- C ABI of the ASL prefill hot path for NVIDIA B200 (sm_100a).
+ *
+ * ASL (adaptive selection layer) watches, layer by layer during prefill, how
+ * the ranking of context tokens by observation-window attention settles, and
+ * prunes the KV cache to a budget.  This library is the per-layer data path:
+ *
+ *   asl_score_layer   Algorithm 1 lines 3-6 + the "scores" sum of Section 4.1
+ *   asl_rank_stat     Algorithm 1 line 9 + Algorithm 2 lines 1-10 (Section 4.1)
+ *   asl_select_topk   Algorithm 1 lines 7-8
+ *   asl_compact_kv    Algorithm 1 line 10
+ *
+ * Conventions
+ *   - Every entry point returns an asl_status; nothing throws, aborts or prints.
+ *   - "device" pointers are CUDA global-memory addresses on the context's
+ *     device; "host" pointers are ordinary process memory.  The caller owns
+ *     every buffer it passes; the library keeps no reference after the call's
+ *     work has finished on the stream.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*);
+ *     no entry point synchronises with the host.
+ *   - The library allocates device memory only inside asl_create/asl_plan
+ *     (a few KB of per-request tables); scratch comes from the caller's
+ *     workspace, whose size asl_plan reports.  The workspace is split into
+ *     disjoint regions per entry point, so asl_rank_stat may run on another
+ *     stream concurrently with asl_select_topk / asl_compact_kv of the same
+ *     layer.  Two calls of the SAME entry point on one context must not overlap.
+ *   - bf16 tensors are passed as raw 16-bit patterns; the channel (head_dim)
+ *     axis is contiguous and every row starts on a 16-byte boundary.
+ *   - Token indices are request-local, 0-based, int32.
+ *   - Requests are packed back to back: request b owns tokens
+ *     [cu_seqlens[b], cu_seqlens[b+1]) of K/V, n_b of them, the last `window`
+ *     being the observation window; T_b = n_b - window past tokens.
+ *     Score vectors are packed the same way over past tokens only: request b's
+ *     segment starts at cu_seqlens[b] - b*window and has T_b entries
+ *     (sum_T in total).  Kept lists are packed over kept_b = min(budget_b, n_b).
+ */
+#ifndef ASL_H_
+#define ASL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct asl_ctx asl_ctx;   /* opaque: plan, device tables, cached tensor maps */
+
+typedef enum {
+  ASL_OK = 0,
+  ASL_ERR_INVALID = -1,      /* bad argument (null, shape, alignment, budget < window ...) */
+  ASL_ERR_UNSUPPORTED = -2,  /* valid request this build cannot run                         */
+  ASL_ERR_WORKSPACE = -3,    /* workspace pointer null or too small                         */
+  ASL_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed                           */
+  ASL_ERR_TIMEOUT = -5,      /* a bounded device-side wait gave up (see asl_device_status)  */
+  ASL_ERR_ARCH = -6          /* device is not sm_100: there is no fallback path             */
+} asl_status;
+
+enum { ASL_POOL_AVG = 0, ASL_POOL_MAX = 1 };
+
+/* Problem statement of Algorithm 1 (W, S, KV_budget) and Algorithm 2
+ * (L_min, L_obs, tau).  Host arrays are copied by asl_plan. */
+typedef struct {
+  int32_t n_q_heads;      /* H_q                                                     */
+  int32_t n_kv_heads;     /* H_k, divides H_q; query head a reads kv head a / G      */
+  int32_t head_dim;       /* d (128 in this build)                                    */
+  int32_t window;         /* W >= 1: observation window = last W query rows           */
+  int32_t pool_kernel;    /* S, odd >= 1; stride 1, pad floor(S/2)                    */
+  int32_t pool_mode;      /* ASL_POOL_AVG (the paper) or ASL_POOL_MAX                 */
+  int32_t batch;          /* B >= 1 requests                                          */
+  int32_t l_min;          /* first layer at which the statistic is evaluated          */
+  int32_t l_obs;          /* rank rows kept (ring depth), >= 2                        */
+  int32_t reserved;
+  double tau;             /* selection fires when relative variance < tau             */
+  const int32_t* cu_seqlens; /* host [B+1] token offsets, cu_seqlens[0] = 0           */
+  const int32_t* budgets;    /* host [B] KV_budget per request, window included       */
+  int64_t q_stride[3];    /* q_obs element strides: request, head, row                */
+  int64_t k_stride[2];    /* K element strides: token, head                           */
+  int64_t v_stride[2];    /* V element strides: token, head                           */
+} asl_params;
+
+/* Result of Algorithm 2 for one request; lives in device memory, [B] of them,
+ * and carries init_var from layer to layer.  Zero it before a new prompt. */
+typedef struct {
+  int64_t num;        /* sum over the union of rows*sum(r^2) - (sum r)^2, exact           */
+  int32_t m;          /* |U|: size of the union of per-row top-k sets                     */
+  int32_t rows;       /* rank rows the statistic was taken over                           */
+  int32_t k;          /* min(KV_budget - W, T)                                            */
+  int32_t layer_idx;  /* layer of the latest call                                         */
+  int32_t evaluated;  /* 1 if layer_idx >= L_min and rows >= 2, else 0 (fields above 0)    */
+  int32_t selected;   /* 1 if rel < tau at this layer                                     */
+  int32_t has_init;   /* init_var holds a value                                           */
+  int32_t reserved;
+  double var_top;     /* num / (rows^2 * m)                                               */
+  double init_var;    /* var_top at the first evaluated layer                             */
+  double rel;         /* var_top / init_var                                               */
+} asl_stat;
+
+/* Context bound to CUDA device `device`.  ASL_ERR_ARCH unless it is sm_100. */
+asl_status asl_create(asl_ctx** out, int device);
+asl_status asl_destroy(asl_ctx* ctx);
+
+/* Validates the parameters, copies the host arrays, builds the per-request
+ * tables on the device and reports the workspace size every later call needs.
+ * ASL_ERR_INVALID for: null pointers, H_q % H_k != 0, even or zero S, W < 1,
+ * n_b <= W (Algorithm 1 needs a non-empty past), budget_b < W, l_obs < 2,
+ * strides that break 16-byte row alignment.  budget_b >= n_b is valid (keep all).
+ * May be called again on the same context to re-plan. */
+asl_status asl_plan(asl_ctx* ctx, const asl_params* params, size_t* workspace_bytes);
+
+/* Derived sizes of the current plan (host values): sum_T = sum of past tokens,
+ * sum_kept = sum of min(budget_b, n_b). */
+asl_status asl_plan_sizes(const asl_ctx* ctx, int64_t* sum_tokens, int64_t* sum_T, int64_t* sum_kept);
+
+/* Algorithm 1 lines 3-6: A = softmax over all n keys of the last W query rows
+ * (causal mask on the last W x W block), U = column sums over the W rows for
+ * past columns, pooled per query head, summed over each GQA group:
+ *   scores_kv  device [H_k][sum_T] fp32   P of Algorithm 1 line 6
+ *   scores_agg device [sum_T]      fp32   sum over kv heads (the "scores" of Section 4.1)
+ * q_obs device bf16 [B][H_q][W][d] (strides q_stride), k device bf16 packed
+ * [sum n_b][H_k][d] (strides k_stride). */
+asl_status asl_score_layer(asl_ctx* ctx, const void* q_obs, const void* k, float* scores_kv,
+                           float* scores_agg, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 1 line 9 + Algorithm 2: writes rank row RankDesc(scores_agg)
+ * (0-based, ties to the lower index) into ring slot layer_idx % L_obs of
+ * rank_ring (device int32 [L_obs][sum_T]), then, if layer_idx >= L_min and
+ * n_rows >= 2, takes the statistic over the latest n_rows rows (the rows of
+ * layers layer_idx-n_rows+1 .. layer_idx, n_rows <= L_obs, this one included):
+ * union of the per-row k smallest ranks, mean population variance of ranks,
+ * relative variance against init_var, comparison with tau.  stat: device [B]. */
+asl_status asl_rank_stat(asl_ctx* ctx, const float* scores_agg, int32_t layer_idx, int32_t n_rows,
+                         int32_t* rank_ring, asl_stat* stat, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* Algorithm 1 lines 7-8 per (request, head): the k_b = min(budget_b, n_b) - W
+ * past tokens with the largest score, ties to the lower index, written in
+ * ascending index order and followed by the window indices T_b .. n_b-1.
+ * scores device [n_heads][sum_T] fp32; idx_out device int32 [n_heads][sum_kept].
+ * n_heads is H_k for the per-head cache, 1 for a selection on the aggregate. */
+asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 1 line 10: k_out[h][r][:] = k[cu_seqlens[b] + idx[h][r]][h][:] and
+ * the same for v, r running over request b's kept segment.
+ * k_out, v_out: device bf16 dense [H_k][sum_kept][d]. */
+asl_status asl_compact_kv(asl_ctx* ctx, const void* k, const void* v, const int32_t* idx, void* k_out,
+                          void* v_out, void* stream);
+
+/* Reads the device error word written by bounded waits (host-synchronising:
+ * it waits for `stream` first).  ASL_OK, or ASL_ERR_TIMEOUT with *where set to
+ * the code of the wait that gave up; the word is cleared. */
+asl_status asl_device_status(asl_ctx* ctx, void* stream, int32_t* where);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t asl_launch_count(const asl_ctx* ctx);
+
+const char* asl_strerror(asl_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASL_H_ */

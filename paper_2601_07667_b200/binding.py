@@ -1,0 +1,259 @@
+"""ctypes binding of libasl_b200.so: same names as the C ABI, argument
+marshalling only.  Every step of the path runs in the library's CUDA kernels;
+PyTorch supplies device memory and streams, nothing else.  There is no CPU
+fallback: a missing library is an ImportError, a failing call an AslError."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libasl_b200.so")
+
+ASL_POOL_AVG, ASL_POOL_MAX = 0, 1
+ASL_OK, ASL_ERR_INVALID, ASL_ERR_UNSUPPORTED, ASL_ERR_WORKSPACE = 0, -1, -2, -3
+ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
+
+EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
+           "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror")
+
+
+class AslParams(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("window", C.c_int32), ("pool_kernel", C.c_int32), ("pool_mode", C.c_int32),
+                ("batch", C.c_int32), ("l_min", C.c_int32), ("l_obs", C.c_int32), ("reserved", C.c_int32),
+                ("tau", C.c_double),
+                ("cu_seqlens", C.POINTER(C.c_int32)), ("budgets", C.POINTER(C.c_int32)),
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 2), ("v_stride", C.c_int64 * 2)]
+
+
+class AslStat(C.Structure):
+    _fields_ = [("num", C.c_int64), ("m", C.c_int32), ("rows", C.c_int32), ("k", C.c_int32),
+                ("layer_idx", C.c_int32), ("evaluated", C.c_int32), ("selected", C.c_int32),
+                ("has_init", C.c_int32), ("reserved", C.c_int32),
+                ("var_top", C.c_double), ("init_var", C.c_double), ("rel", C.c_double)]
+
+
+STAT_DTYPE = np.dtype([("num", "<i8"), ("m", "<i4"), ("rows", "<i4"), ("k", "<i4"), ("layer_idx", "<i4"),
+                       ("evaluated", "<i4"), ("selected", "<i4"), ("has_init", "<i4"), ("reserved", "<i4"),
+                       ("var_top", "<f8"), ("init_var", "<f8"), ("rel", "<f8")])
+assert STAT_DTYPE.itemsize == C.sizeof(AslStat) == 64
+
+
+class AslError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {asl_strerror(status)} ({status})")
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_07667_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    lib.asl_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.asl_destroy.argtypes = [vp]
+    lib.asl_plan.argtypes = [vp, C.POINTER(AslParams), C.POINTER(sz)]
+    lib.asl_plan_sizes.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
+    lib.asl_score_layer.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.asl_rank_stat.argtypes = [vp, vp, i32, i32, vp, vp, vp, sz, vp]
+    lib.asl_select_topk.argtypes = [vp, vp, i32, vp, vp, sz, vp]
+    lib.asl_compact_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.asl_device_status.argtypes = [vp, vp, C.POINTER(i32)]
+    lib.asl_launch_count.argtypes = [vp]
+    lib.asl_launch_count.restype = i64
+    lib.asl_strerror.argtypes = [C.c_int]
+    lib.asl_strerror.restype = C.c_char_p
+    for name in EXPORTS:
+        if name not in ("asl_launch_count", "asl_strerror"):
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def library() -> C.CDLL:
+    return _lib
+
+
+def asl_strerror(status: int) -> str:
+    return _lib.asl_strerror(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != ASL_OK:
+        raise AslError(status, what)
+
+
+def _ptr(x) -> int:
+    """Device (or host) address of a torch tensor / raw integer address."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+# ---- the C entry points, one Python function each ---------------------------------
+def asl_create(device: int = 0) -> int:
+    h = C.c_void_p()
+    _check(_lib.asl_create(C.byref(h), int(device)), "asl_create")
+    return h.value
+
+
+def asl_destroy(ctx: int) -> None:
+    _check(_lib.asl_destroy(ctx), "asl_destroy")
+
+
+def asl_plan(ctx: int, *, n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, pool_kernel: int,
+             pool_mode: int, cu_seqlens: Sequence[int], budgets: Sequence[int], l_min: int, l_obs: int,
+             tau: float, q_stride: Sequence[int], k_stride: Sequence[int], v_stride: Sequence[int]) -> int:
+    cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    bu = (C.c_int32 * len(budgets))(*[int(x) for x in budgets])
+    p = AslParams(n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, len(budgets), l_min, l_obs, 0,
+                  float(tau), cu, bu, (C.c_int64 * 3)(*q_stride), (C.c_int64 * 2)(*k_stride),
+                  (C.c_int64 * 2)(*v_stride))
+    if len(cu_seqlens) != len(budgets) + 1:
+        raise AslError(ASL_ERR_INVALID, "asl_plan")
+    size = C.c_size_t(0)
+    _check(_lib.asl_plan(ctx, C.byref(p), C.byref(size)), "asl_plan")
+    return size.value
+
+
+def asl_plan_sizes(ctx: int):
+    a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(_lib.asl_plan_sizes(ctx, C.byref(a), C.byref(b), C.byref(c)), "asl_plan_sizes")
+    return a.value, b.value, c.value
+
+
+def asl_score_layer(ctx, q_obs, k, scores_kv, scores_agg, workspace, workspace_bytes, stream=None) -> None:
+    _check(_lib.asl_score_layer(ctx, _ptr(q_obs), _ptr(k), _ptr(scores_kv), _ptr(scores_agg), _ptr(workspace),
+                                int(workspace_bytes), _stream_handle(stream)), "asl_score_layer")
+
+
+def asl_rank_stat(ctx, scores_agg, layer_idx, n_rows, rank_ring, stat, workspace, workspace_bytes, stream=None) -> None:
+    _check(_lib.asl_rank_stat(ctx, _ptr(scores_agg), int(layer_idx), int(n_rows), _ptr(rank_ring), _ptr(stat),
+                              _ptr(workspace), int(workspace_bytes), _stream_handle(stream)), "asl_rank_stat")
+
+
+def asl_select_topk(ctx, scores, n_heads, idx_out, workspace, workspace_bytes, stream=None) -> None:
+    _check(_lib.asl_select_topk(ctx, _ptr(scores), int(n_heads), _ptr(idx_out), _ptr(workspace),
+                                int(workspace_bytes), _stream_handle(stream)), "asl_select_topk")
+
+
+def asl_compact_kv(ctx, k, v, idx, k_out, v_out, stream=None) -> None:
+    _check(_lib.asl_compact_kv(ctx, _ptr(k), _ptr(v), _ptr(idx), _ptr(k_out), _ptr(v_out),
+                               _stream_handle(stream)), "asl_compact_kv")
+
+
+def asl_device_status(ctx, stream=None):
+    where = C.c_int32(0)
+    st = _lib.asl_device_status(ctx, _stream_handle(stream), C.byref(where))
+    return st, where.value
+
+
+def asl_launch_count(ctx) -> int:
+    return int(_lib.asl_launch_count(ctx))
+
+
+# ---- a small holder of one plan's device buffers -------------------------------------
+class LayerPath:
+    """Owns a context, its plan and the device buffers of one layer's pass
+    (scores, indices, compacted cache, rank ring, statistic), all torch tensors.
+    ``run_layer`` issues the five steps; the rank statistic goes to a side stream
+    so it overlaps the top-k and the compaction."""
+
+    def __init__(self, *, n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, seqlens, budgets,
+                 l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None):
+        import torch
+        self.torch = torch
+        self.dev = torch.device("cuda", device)
+        self.ctx = asl_create(device)
+        self.H_q, self.H_k, self.d, self.w = n_q_heads, n_kv_heads, head_dim, window
+        self.l_min, self.l_obs = l_min, l_obs
+        self.seqlens = [int(n) for n in seqlens]
+        self.batch = len(self.seqlens)
+        cu = np.concatenate([[0], np.cumsum(self.seqlens)]).astype(np.int64)
+        self.cu = cu
+        q_stride = q_stride or (n_q_heads * window * head_dim, window * head_dim, head_dim)
+        k_stride = k_stride or (n_kv_heads * head_dim, head_dim)
+        v_stride = v_stride or (n_kv_heads * head_dim, head_dim)
+        self.ws_bytes = asl_plan(self.ctx, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
+                                 window=window, pool_kernel=pool_kernel, pool_mode=pool_mode, cu_seqlens=cu,
+                                 budgets=budgets, l_min=l_min, l_obs=l_obs, tau=tau, q_stride=q_stride,
+                                 k_stride=k_stride, v_stride=v_stride)
+        self.sum_tokens, self.sum_T, self.sum_kept = asl_plan_sizes(self.ctx)
+        self.kept = [min(int(bg), n) for bg, n in zip(budgets, self.seqlens)]
+        self.t_off = np.concatenate([[0], np.cumsum([n - window for n in self.seqlens])]).astype(np.int64)
+        self.kept_off = np.concatenate([[0], np.cumsum(self.kept)]).astype(np.int64)
+        dev = self.dev
+        self.workspace = torch.empty(max(self.ws_bytes, 256), dtype=torch.uint8, device=dev)
+        self.scores_kv = torch.empty((n_kv_heads, self.sum_T), dtype=torch.float32, device=dev)
+        self.scores_agg = torch.empty((self.sum_T,), dtype=torch.float32, device=dev)
+        self.idx = torch.empty((n_kv_heads, self.sum_kept), dtype=torch.int32, device=dev)
+        self.k_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
+        self.v_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
+        self.rank_ring = torch.zeros((l_obs, self.sum_T), dtype=torch.int32, device=dev)
+        self.stat = torch.zeros((self.batch, C.sizeof(AslStat)), dtype=torch.uint8, device=dev)
+        self.side = torch.cuda.Stream(device=dev)
+        self._fork = torch.cuda.Event()
+        self._join = torch.cuda.Event()
+        self.first_layer: Optional[int] = None
+
+    def close(self) -> None:
+        if self.ctx:
+            asl_destroy(self.ctx)
+            self.ctx = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self) -> None:
+        """New prompt: forget init_var and the rank rows."""
+        self.stat.zero_()
+        self.first_layer = None
+
+    def n_rows(self, layer_idx: int) -> int:
+        if self.first_layer is None:
+            self.first_layer = layer_idx
+        return min(self.l_obs, layer_idx - self.first_layer + 1)
+
+    def run_layer(self, q_obs, k, v, layer_idx: int, *, overlap: bool = True) -> None:
+        """Steps a1..a5 for one layer on the current stream (statistic on the side stream)."""
+        torch = self.torch
+        ctx, ws, wsb = self.ctx, self.workspace, self.ws_bytes
+        rows = self.n_rows(layer_idx)
+        asl_score_layer(ctx, q_obs, k, self.scores_kv, self.scores_agg, ws, wsb)
+        if overlap:
+            main = torch.cuda.current_stream()
+            self._fork.record(main)
+            self.side.wait_event(self._fork)
+            asl_rank_stat(ctx, self.scores_agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, self.side)
+            self._join.record(self.side)
+        else:
+            asl_rank_stat(ctx, self.scores_agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb)
+        asl_select_topk(ctx, self.scores_kv, self.H_k, self.idx, ws, wsb)
+        asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out)
+        if overlap:
+            torch.cuda.current_stream().wait_event(self._join)
+
+    def read_stat(self) -> np.ndarray:
+        """Device -> host copy of the [B] statistic records (synchronises)."""
+        return self.stat.cpu().numpy().view(STAT_DTYPE).reshape(self.batch)

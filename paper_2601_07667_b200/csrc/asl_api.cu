@@ -1,0 +1,209 @@
+// C-ABI entry points: argument checks, planning, workspace layout, dispatch.
+#include <math.h>
+#include <new>
+
+#include "asl_internal.cuh"
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void free_plan(asl_ctx* c) {
+  if (c->d_req) cudaFree(c->d_req);
+  if (c->d_acc) cudaFree(c->d_acc);
+  c->d_req = nullptr;
+  c->d_acc = nullptr;
+  c->planned = false;
+}
+
+}  // namespace
+
+extern "C" {
+
+asl_status asl_create(asl_ctx** out, int device) {
+  if (!out) return ASL_ERR_INVALID;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return ASL_ERR_CUDA;
+  cudaDeviceProp prop;
+  ASL_CUDA(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return ASL_ERR_ARCH;      // sm_100 only: no fallback path
+  asl_ctx* c = new (std::nothrow) asl_ctx();
+  if (!c) return ASL_ERR_CUDA;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(device);
+  cudaError_t e = cudaMalloc(&c->d_err, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(c->d_err, 0, sizeof(int32_t));
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) { delete c; return ASL_ERR_CUDA; }
+  *out = c;
+  return ASL_OK;
+}
+
+asl_status asl_destroy(asl_ctx* c) {
+  if (!c) return ASL_ERR_INVALID;
+  free_plan(c);
+  if (c->d_err) cudaFree(c->d_err);
+  delete c;
+  return ASL_OK;
+}
+
+asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
+  if (!c || !p || !workspace_bytes || !p->cu_seqlens || !p->budgets) return ASL_ERR_INVALID;
+  if (p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return ASL_ERR_INVALID;
+  if (p->window < 1 || p->batch < 1) return ASL_ERR_INVALID;
+  if (p->pool_kernel < 1 || p->pool_kernel % 2 == 0) return ASL_ERR_INVALID;
+  if (p->pool_mode != ASL_POOL_AVG && p->pool_mode != ASL_POOL_MAX) return ASL_ERR_INVALID;
+  if (p->l_obs < 2 || p->l_min < 0) return ASL_ERR_INVALID;
+  if (p->head_dim < 8 || p->head_dim % 8) return ASL_ERR_INVALID;
+  if (p->head_dim != 128) return ASL_ERR_UNSUPPORTED;
+  // rows must start on 16-byte boundaries: every stride a multiple of 8 elements
+  const int64_t strides[] = {p->q_stride[0], p->q_stride[1], p->q_stride[2], p->k_stride[0],
+                             p->k_stride[1], p->v_stride[0], p->v_stride[1]};
+  for (int64_t s : strides)
+    if (s < 0 || s % 8) return ASL_ERR_INVALID;
+  if (p->q_stride[2] < p->head_dim || p->k_stride[1] < p->head_dim || p->v_stride[1] < p->head_dim) return ASL_ERR_INVALID;
+  if (p->cu_seqlens[0] != 0) return ASL_ERR_INVALID;
+
+  std::vector<AslReq> req(p->batch);
+  int64_t sum_T = 0, sum_kept = 0, tiles = 0;
+  int32_t max_n = 0, max_T = 0, max_kept = 0;
+  for (int b = 0; b < p->batch; ++b) {
+    const int64_t n = (int64_t)p->cu_seqlens[b + 1] - p->cu_seqlens[b];
+    const int64_t budget = p->budgets[b];
+    if (n <= p->window || budget < p->window) return ASL_ERR_INVALID;
+    AslReq& r = req[b];
+    r.n = (int32_t)n;
+    r.T = (int32_t)(n - p->window);
+    r.kept = (int32_t)(budget < n ? budget : n);
+    r.k = r.kept - p->window;
+    r.tok_off = p->cu_seqlens[b];
+    r.t_off = (int32_t)sum_T;
+    r.kept_off = (int32_t)sum_kept;
+    r.pad = (int32_t)tiles;                       // first key tile of the request (SIMT scorer partials)
+    sum_T += r.T;
+    sum_kept += r.kept;
+    tiles += (n + ASL_SIMT_KEY_TILE - 1) / ASL_SIMT_KEY_TILE;
+    max_n = r.n > max_n ? r.n : max_n;
+    max_T = r.T > max_T ? r.T : max_T;
+    max_kept = r.kept > max_kept ? r.kept : max_kept;
+    // the integer numerator of the statistic must fit 63 bits: m * rows^2 * T^2 / 4
+    const double m_max = fmin((double)r.T, (double)(r.k > 0 ? r.k : 1) * p->l_obs);
+    if (m_max * p->l_obs * p->l_obs * (double)r.T * (double)r.T / 4.0 >= 9.0e18) return ASL_ERR_UNSUPPORTED;
+  }
+  if (sum_T >= (int64_t)1 << 31 || (int64_t)p->cu_seqlens[p->batch] >= (int64_t)1 << 31) return ASL_ERR_UNSUPPORTED;
+
+  int prev = 0;
+  cudaGetDevice(&prev);
+  ASL_CUDA(cudaSetDevice(c->device));
+  free_plan(c);
+  cudaError_t e = cudaMalloc(&c->d_req, sizeof(AslReq) * p->batch);
+  if (e == cudaSuccess) e = cudaMemcpy(c->d_req, req.data(), sizeof(AslReq) * p->batch, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_acc, sizeof(unsigned long long) * 2 * p->batch);
+  if (e == cudaSuccess) e = cudaMemset(c->d_acc, 0, sizeof(unsigned long long) * 2 * p->batch);
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) { free_plan(c); return ASL_ERR_CUDA; }
+
+  c->p = *p;
+  c->cu.assign(p->cu_seqlens, p->cu_seqlens + p->batch + 1);
+  c->budgets.assign(p->budgets, p->budgets + p->batch);
+  c->p.cu_seqlens = c->cu.data();
+  c->p.budgets = c->budgets.data();
+  c->req = req;
+  c->sum_tokens = p->cu_seqlens[p->batch];
+  c->sum_T = sum_T;
+  c->sum_kept = sum_kept;
+  c->max_n = max_n; c->max_T = max_T; c->max_kept = max_kept;
+  c->rows_per_kv = (p->n_q_heads / p->n_kv_heads) * p->window;
+  c->n_key_tiles = (int32_t)tiles;
+
+  AslWorkspace& w = c->ws;
+  size_t off = 0;
+  w.score_partials = off; off = asl_align256(off + (size_t)tiles * p->n_kv_heads * c->rows_per_kv * sizeof(float2));
+  w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * c->rows_per_kv * sizeof(float));
+  const size_t u_rows = p->pool_mode == ASL_POOL_MAX ? p->n_q_heads : p->n_kv_heads;
+  w.score_u = off;        off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float));
+  w.score_end = off;
+  for (int i = 0; i < 2; ++i) { w.rank_keys[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
+  for (int i = 0; i < 2; ++i) { w.rank_idx[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
+  const size_t nblk = (max_T + ASL_RANK_TILE - 1) / ASL_RANK_TILE;
+  w.rank_hist = off;      off = asl_align256(off + (size_t)p->batch * 256 * nblk * sizeof(int32_t));
+  w.rank_end = off;
+  w.topk_end = off;
+  w.total = off;
+  *workspace_bytes = w.total;
+  c->planned = true;
+  return ASL_OK;
+}
+
+asl_status asl_plan_sizes(const asl_ctx* c, int64_t* sum_tokens, int64_t* sum_T, int64_t* sum_kept) {
+  if (!c || !c->planned) return ASL_ERR_INVALID;
+  if (sum_tokens) *sum_tokens = c->sum_tokens;
+  if (sum_T) *sum_T = c->sum_T;
+  if (sum_kept) *sum_kept = c->sum_kept;
+  return ASL_OK;
+}
+
+asl_status asl_score_layer(asl_ctx* c, const void* q_obs, const void* k, float* scores_kv, float* scores_agg,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  if (!c || !c->planned || !q_obs || !k || !scores_kv || !scores_agg) return ASL_ERR_INVALID;
+  if (!aligned16(q_obs) || !aligned16(k)) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  return asl_launch_score_simt(c, q_obs, k, scores_kv, scores_agg, static_cast<char*>(workspace),
+                               static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_rank_stat(asl_ctx* c, const float* scores_agg, int32_t layer_idx, int32_t n_rows, int32_t* rank_ring,
+                         asl_stat* stat, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!c || !c->planned || !scores_agg || !rank_ring || !stat) return ASL_ERR_INVALID;
+  if (layer_idx < 0 || n_rows < 1 || n_rows > c->p.l_obs || n_rows > layer_idx + 1) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  return asl_launch_rank(c, scores_agg, layer_idx, n_rows, rank_ring, stat, static_cast<char*>(workspace),
+                         static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_select_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  if (!c || !c->planned || !scores || !idx_out || n_heads < 1) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total) return ASL_ERR_WORKSPACE;
+  return asl_launch_topk(c, scores, n_heads, idx_out, static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_compact_kv(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
+                          void* stream) {
+  if (!c || !c->planned || !k || !v || !idx || !k_out || !v_out) return ASL_ERR_INVALID;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out)) return ASL_ERR_INVALID;
+  return asl_launch_compact(c, k, v, idx, k_out, v_out, static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_device_status(asl_ctx* c, void* stream, int32_t* where) {
+  if (!c) return ASL_ERR_INVALID;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t word = 0;
+  ASL_CUDA(cudaMemcpyAsync(&word, c->d_err, sizeof(word), cudaMemcpyDeviceToHost, st));
+  ASL_CUDA(cudaStreamSynchronize(st));
+  if (where) *where = word;
+  if (word == 0) return ASL_OK;
+  ASL_CUDA(cudaMemsetAsync(c->d_err, 0, sizeof(word), st));
+  return ASL_ERR_TIMEOUT;
+}
+
+int64_t asl_launch_count(const asl_ctx* c) { return c ? c->launches : 0; }
+
+const char* asl_strerror(asl_status s) {
+  switch (s) {
+    case ASL_OK: return "ok";
+    case ASL_ERR_INVALID: return "invalid argument";
+    case ASL_ERR_UNSUPPORTED: return "unsupported configuration";
+    case ASL_ERR_WORKSPACE: return "workspace missing or too small";
+    case ASL_ERR_CUDA: return "CUDA call failed";
+    case ASL_ERR_TIMEOUT: return "bounded device wait expired";
+    case ASL_ERR_ARCH: return "device is not sm_100";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

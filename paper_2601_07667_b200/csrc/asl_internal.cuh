@@ -1,0 +1,75 @@
+// Internal declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <vector>
+
+#include "asl.h"
+
+// Per-request table entry, one per request, resident on the device.
+struct AslReq {
+  int32_t n;         // tokens, window included
+  int32_t T;         // past tokens n - W
+  int32_t k;         // past tokens kept: min(budget, n) - W
+  int32_t kept;      // k + W
+  int32_t tok_off;   // cu_seqlens[b]
+  int32_t t_off;     // offset of the request's past segment in packed score vectors
+  int32_t kept_off;  // offset of the request's segment in packed kept lists
+  int32_t pad;
+};
+
+// Scratch layout inside the caller's workspace (byte offsets, 256-aligned).
+struct AslWorkspace {
+  size_t score_partials;   // pass-1 partial row statistics
+  size_t score_offsets;    // per-row log2 normalisers
+  size_t score_u;          // un-pooled column sums
+  size_t score_end;
+  size_t rank_keys[2];     // ping-pong sort keys
+  size_t rank_idx[2];      // ping-pong sort payload
+  size_t rank_hist;        // per-block digit histograms / offsets
+  size_t rank_end;
+  size_t topk_end;         // (top-k keeps its state on chip)
+  size_t total;
+};
+
+struct asl_ctx {
+  int device = 0;
+  int sm_count = 0;
+  bool planned = false;
+  asl_params p{};
+  std::vector<int32_t> cu, budgets;
+  std::vector<AslReq> req;
+  int64_t sum_tokens = 0, sum_T = 0, sum_kept = 0;
+  int32_t max_n = 0, max_T = 0, max_kept = 0;
+  AslReq* d_req = nullptr;            // device [B]
+  unsigned long long* d_acc = nullptr;  // device [B][2] integer accumulators of the statistic
+  int32_t* d_err = nullptr;           // device error word of bounded waits
+  // scorer plan
+  int32_t rows_per_kv = 0;            // G*W
+  int32_t n_key_tiles = 0;            // sum over requests of ceil(n_b / tile)
+  int32_t p1_splits = 0;              // partials per row written by pass 1
+  AslWorkspace ws{};
+  int64_t launches = 0;
+};
+
+#define ASL_CUDA(expr)                          \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return ASL_ERR_CUDA; \
+  } while (0)
+
+static inline size_t asl_align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+// ---- kernels' host launchers (one per translation unit) ----
+asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
+                                 char* ws, cudaStream_t st);
+asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
+asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
+                           asl_stat* stat, char* ws, cudaStream_t st);
+asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, cudaStream_t st);
+asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
+                              cudaStream_t st);
+
+constexpr int ASL_SIMT_KEY_TILE = 128;   // keys per block in the SIMT scorer
+constexpr int ASL_RANK_TILE = 4096;      // keys per block in the radix sort

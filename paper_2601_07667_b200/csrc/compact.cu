@@ -1,0 +1,41 @@
+// K/V compaction (Algorithm 1 line 10): out[h][r][:] = x[tok_off + idx[h][r]][h][:].
+// 16 threads move one 256-byte row as 16-byte vectors; K and V in one launch.
+#include "asl_internal.cuh"
+
+namespace {
+
+__global__ void __launch_bounds__(256) compact_kv_kernel(const uint16_t* __restrict__ k, const uint16_t* __restrict__ v,
+                                                         const int32_t* __restrict__ idx, const AslReq* __restrict__ req,
+                                                         int64_t ks_t, int64_t ks_h, int64_t vs_t, int64_t vs_h,
+                                                         int64_t sum_kept, int vec_per_row, uint16_t* __restrict__ k_out,
+                                                         uint16_t* __restrict__ v_out) {
+  const int b = blockIdx.z, h = blockIdx.y;
+  const AslReq rq = req[b];
+  const int rows_per_block = blockDim.x / vec_per_row;
+  const int r = blockIdx.x * rows_per_block + threadIdx.x / vec_per_row;
+  const int c = threadIdx.x % vec_per_row;
+  if (r >= rq.kept) return;
+  const int64_t orow = (int64_t)h * sum_kept + rq.kept_off + r;
+  const int64_t tok = (int64_t)rq.tok_off + idx[orow];
+  const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * ks_t + (int64_t)h * ks_h + c * 8);
+  const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * vs_t + (int64_t)h * vs_h + c * 8);
+  const int64_t o = orow * (vec_per_row * 8) + c * 8;
+  *reinterpret_cast<uint4*>(k_out + o) = kv;
+  *reinterpret_cast<uint4*>(v_out + o) = vv;
+}
+
+}  // namespace
+
+asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
+                              cudaStream_t st) {
+  const asl_params& p = c->p;
+  const int vec = p.head_dim / 8;                 // 16-byte vectors per row
+  const int rows_per_block = 256 / vec;
+  dim3 grid((c->max_kept + rows_per_block - 1) / rows_per_block, p.n_kv_heads, p.batch);
+  compact_kv_kernel<<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), idx, c->d_req,
+                                          p.k_stride[0], p.k_stride[1], p.v_stride[0], p.v_stride[1], c->sum_kept, vec,
+                                          static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out));
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}

@@ -1,0 +1,246 @@
+// Rank row and rank-variance statistic (Algorithm 1 line 9; Algorithm 2 lines 5-10;
+// Section 4.1 "var_top" and "relative variance").
+//
+// RankDesc: stable least-significant-digit radix sort (8-bit digits) of
+// (key, token index) pairs per request, key = bit pattern that ascends as the
+// score descends; equal scores keep ascending index order, so the position of
+// a token in the sorted sequence is its 0-based rank with ties to the lower
+// index.  The last pass scatters positions straight into the ring row.
+//
+// Statistic: a token is in the union iff its smallest rank over the rows is < k
+// (the k smallest ranks of a row are exactly ranks 0..k-1).  The numerator
+// sum_j (rows*sum r^2 - (sum r)^2) is accumulated in 64-bit integers with
+// integer atomics, so it does not depend on the order of accumulation.
+#include "asl_internal.cuh"
+
+namespace {
+
+constexpr int TILE = ASL_RANK_TILE;
+constexpr int SORT_THREADS = 256;
+constexpr int WARPS = SORT_THREADS / 32;
+constexpr int PER_WARP = TILE / WARPS;   // 512 keys, walked 32 at a time
+
+__device__ __forceinline__ uint32_t desc_key(float s) {
+  uint32_t u = __float_as_uint(s);
+  if (u == 0x80000000u) u = 0;                           // -0 ranks with +0
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);        // ascending with the score
+  return ~u;                                             // ascending as the score descends
+}
+
+__global__ void rank_prepare(const float* __restrict__ agg, const AslReq* __restrict__ req, uint32_t* __restrict__ keys,
+                             int32_t* __restrict__ idx) {
+  const AslReq rq = req[blockIdx.y];
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= rq.T) return;
+  keys[rq.t_off + j] = desc_key(agg[rq.t_off + j]);
+  idx[rq.t_off + j] = j;
+}
+
+// hist[b][digit][blk]: digit counts of one tile
+__global__ void __launch_bounds__(SORT_THREADS) rank_hist(const uint32_t* __restrict__ keys, const AslReq* __restrict__ req,
+                                                          int shift, int nblk, int32_t* __restrict__ hist) {
+  __shared__ int cnt[256];
+  const int b = blockIdx.y, blk = blockIdx.x;
+  const AslReq rq = req[b];
+  cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const int start = blk * TILE;
+  if (start < rq.T) {
+    const int end = min(rq.T, start + TILE);
+    for (int i = start + threadIdx.x; i < end; i += SORT_THREADS)
+      atomicAdd(&cnt[(keys[rq.t_off + i] >> shift) & 255], 1);
+  }
+  __syncthreads();
+  hist[((int64_t)b * 256 + threadIdx.x) * nblk + blk] = cnt[threadIdx.x];
+}
+
+// exclusive scan of hist[b] in (digit, blk) order, in place
+__global__ void __launch_bounds__(256) rank_scan(int32_t* __restrict__ hist, int nblk) {
+  __shared__ int warp_tot[8];
+  int32_t* row = hist + ((int64_t)blockIdx.x * 256 + threadIdx.x) * nblk;
+  int total = 0;
+  for (int i = 0; i < nblk; ++i) total += row[i];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  int incl = total;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_tot[wid] = incl;
+  __syncthreads();
+  int base = incl - total;
+  for (int w2 = 0; w2 < wid; ++w2) base += warp_tot[w2];
+  for (int i = 0; i < nblk; ++i) {
+    int v = row[i];
+    row[i] = base;
+    base += v;
+  }
+}
+
+// stable scatter of one tile; on the last pass writes rank[token] = position
+__global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const uint32_t* __restrict__ keys_in,
+                                                             const int32_t* __restrict__ idx_in,
+                                                             uint32_t* __restrict__ keys_out, int32_t* __restrict__ idx_out,
+                                                             int32_t* __restrict__ rank_row, const int32_t* __restrict__ offs,
+                                                             const AslReq* __restrict__ req, int shift, int nblk) {
+  __shared__ int cnt[WARPS][256];
+  const int b = blockIdx.y, blk = blockIdx.x;
+  const AslReq rq = req[b];
+  const int start = blk * TILE;
+  if (start >= rq.T) return;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&cnt[0][0])[i] = 0;
+  __syncthreads();
+  const int wstart = start + wid * PER_WARP;
+  const uint32_t lt = (1u << lane) - 1u;
+  // per-warp digit counts
+  for (int r = 0; r < PER_WARP / 32; ++r) {
+    const int i = wstart + r * 32 + lane;
+    const bool valid = i < rq.T;
+    const uint32_t key = valid ? keys_in[rq.t_off + i] : 0u;
+    const int d = valid ? (int)((key >> shift) & 255) : (256 + lane);
+    const uint32_t peers = __match_any_sync(0xffffffffu, d);
+    if (valid && (peers & lt) == 0) cnt[wid][d] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  {  // digit threadIdx.x: bases of the warps, in warp order, after the tile's global offset
+    int run = offs[((int64_t)b * 256 + threadIdx.x) * nblk + blk];
+#pragma unroll
+    for (int w2 = 0; w2 < WARPS; ++w2) {
+      int v = cnt[w2][threadIdx.x];
+      cnt[w2][threadIdx.x] = run;
+      run += v;
+    }
+  }
+  __syncthreads();
+  for (int r = 0; r < PER_WARP / 32; ++r) {
+    const int i = wstart + r * 32 + lane;
+    const bool valid = i < rq.T;
+    const uint32_t key = valid ? keys_in[rq.t_off + i] : 0u;
+    const int32_t id = valid ? idx_in[rq.t_off + i] : 0;
+    const int d = valid ? (int)((key >> shift) & 255) : (256 + lane);
+    const uint32_t peers = __match_any_sync(0xffffffffu, d);
+    int pos = 0;
+    if (valid) pos = cnt[wid][d] + __popc(peers & lt);
+    __syncwarp();
+    if (valid && (peers & lt) == 0) cnt[wid][d] += __popc(peers);
+    __syncwarp();
+    if (valid) {
+      if (rank_row) rank_row[rq.t_off + id] = pos;
+      else { keys_out[rq.t_off + pos] = key; idx_out[rq.t_off + pos] = id; }
+    }
+  }
+}
+
+struct StatArgs {
+  const int32_t* ring;
+  const AslReq* req;
+  unsigned long long* acc;   // [B][2]: numerator, union size
+  int64_t sum_T;
+  int32_t l_obs, first_layer, n_rows;
+};
+
+__global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
+  __shared__ unsigned long long s_num[8];
+  __shared__ int s_m[8];
+  const int b = blockIdx.y;
+  const AslReq rq = a.req[b];
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  unsigned long long num = 0;
+  int m = 0;
+  if (j < rq.T) {
+    long long s1 = 0, s2 = 0;
+    int mn = 0x7fffffff;
+    for (int r = 0; r < a.n_rows; ++r) {
+      const int slot = (a.first_layer + r) % a.l_obs;
+      const long long v = a.ring[(int64_t)slot * a.sum_T + rq.t_off + j];
+      mn = min(mn, (int)v);
+      s1 += v;
+      s2 += v * v;
+    }
+    if (mn < rq.k) {
+      m = 1;
+      num = (unsigned long long)((long long)a.n_rows * s2 - s1 * s1);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    num += __shfl_down_sync(0xffffffffu, num, o);
+    m += __shfl_down_sync(0xffffffffu, m, o);
+  }
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (lane == 0) { s_num[wid] = num; s_m[wid] = m; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w2 = 1; w2 < 8; ++w2) { num += s_num[w2]; m += s_m[w2]; }
+    if (m) {
+      atomicAdd(&a.acc[2 * b], num);
+      atomicAdd(&a.acc[2 * b + 1], (unsigned long long)m);
+    }
+  }
+}
+
+__global__ void rank_stat_finalize(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat,
+                                   int batch, int layer_idx, int n_rows, int evaluate, double tau) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  asl_stat s = stat[b];
+  s.layer_idx = layer_idx;
+  s.k = req[b].k;
+  s.rows = n_rows;
+  s.evaluated = 0;
+  s.selected = 0;
+  s.num = 0;
+  s.m = 0;
+  if (evaluate) {
+    const unsigned long long num = acc[2 * b], m = acc[2 * b + 1];
+    acc[2 * b] = 0;
+    acc[2 * b + 1] = 0;
+    s.num = (int64_t)num;
+    s.m = (int32_t)m;
+    s.evaluated = 1;
+    s.var_top = (double)num / ((double)n_rows * (double)n_rows * (double)m);   // empty union (k = 0): NaN, never selects
+    if (!s.has_init) { s.init_var = s.var_top; s.has_init = 1; }
+    s.rel = s.var_top / s.init_var;
+    s.selected = (s.rel < tau) ? 1 : 0;
+  }
+  stat[b] = s;
+}
+
+}  // namespace
+
+asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
+                           asl_stat* stat, char* ws, cudaStream_t st) {
+  const asl_params& p = c->p;
+  uint32_t* keys[2] = {reinterpret_cast<uint32_t*>(ws + c->ws.rank_keys[0]),
+                       reinterpret_cast<uint32_t*>(ws + c->ws.rank_keys[1])};
+  int32_t* idx[2] = {reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[0]),
+                     reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[1])};
+  int32_t* hist = reinterpret_cast<int32_t*>(ws + c->ws.rank_hist);
+  const int nblk = (c->max_T + TILE - 1) / TILE;
+  int32_t* row = ring + (int64_t)(layer_idx % p.l_obs) * c->sum_T;
+  rank_prepare<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(agg, c->d_req, keys[0], idx[0]);
+  c->launches += 1;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int in = pass & 1, out = in ^ 1;
+    const int shift = pass * 8;
+    rank_hist<<<dim3(nblk, p.batch), SORT_THREADS, 0, st>>>(keys[in], c->d_req, shift, nblk, hist);
+    rank_scan<<<p.batch, 256, 0, st>>>(hist, nblk);
+    rank_scatter<<<dim3(nblk, p.batch), SORT_THREADS, 0, st>>>(keys[in], idx[in], keys[out], idx[out],
+                                                               pass == 3 ? row : nullptr, hist, c->d_req, shift, nblk);
+    c->launches += 3;
+  }
+  const int evaluate = (layer_idx >= p.l_min && n_rows >= 2) ? 1 : 0;
+  if (evaluate) {
+    StatArgs a{ring, c->d_req, c->d_acc, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows};
+    rank_stat_accumulate<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(a);
+    c->launches += 1;
+  }
+  rank_stat_finalize<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, evaluate,
+                                                         p.tau);
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}

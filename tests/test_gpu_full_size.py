@@ -1,0 +1,57 @@
+"""GPU parity at the benchmark's full sizes (the five named workloads), in the
+launch configuration bench.py times.  The oracle computes whole layers here
+(seconds each on the host), so the comparison stays element by element; the
+number of layers is bounded to keep the suite within minutes."""
+import numpy as np
+import pytest
+
+from paper_2601_07667_b200 import inputs as I
+
+from asl_check import StatReplay, check_layer, make_path
+
+pytestmark = pytest.mark.gpu
+
+
+def sweep(wl, seed, layers):
+    path = make_path(wl)
+    replay = StatReplay(wl)
+    rel_gpu, rel_ref = {}, {}
+    for layer in layers:
+        x = I.layer_inputs(wl, layer, seed)
+        res = check_layer(path, wl, x, layer)
+        iso, e2e = replay.step(path, layer, res)[0]
+        if iso["evaluated"]:
+            rel_gpu[layer], rel_ref[layer] = iso["rel"], e2e["rel"]
+    sel_gpu = [c.selected_layer for c in replay.on_gpu_scores]
+    sel_ref = [c.selected_layer for c in replay.on_ref_scores]
+    path.close()
+    return rel_gpu, rel_ref, sel_gpu, sel_ref
+
+
+def test_c2_layer_sweep_selects_the_same_layer():
+    wl = I.workload("C2")
+    first = wl.l_min - wl.l_obs + 1                        # ring is full when the statistic starts
+    rel_gpu, rel_ref, sel_gpu, sel_ref = sweep(wl, 0, range(first, wl.layers))
+    assert sel_gpu == sel_ref
+    assert first < sel_ref[0] < wl.layers - 1               # crosses the threshold mid-stack
+    ls = sorted(rel_ref)
+    assert min(ls, key=lambda l: rel_gpu[l]) == min(ls, key=lambda l: rel_ref[l])
+    dev = max(abs(rel_gpu[l] - rel_ref[l]) for l in ls)
+    margin = min(abs(rel_ref[l] - wl.tau) for l in ls)
+    assert margin >= 10 * dev, f"threshold margin {margin:.4f} vs GPU/oracle deviation {dev:.5f}"
+
+
+def test_c3_long_context_layers():
+    wl = I.workload("C3")
+    rel_gpu, rel_ref, sel_gpu, sel_ref = sweep(wl, 0, range(0, 4))
+    assert sel_gpu == sel_ref
+
+
+def test_c4_ragged_batch_full():
+    wl = I.workload("C4", seed=0)
+    sweep(wl, 0, range(0, 2))
+
+
+def test_c5_wide_gqa_max_pool_full():
+    wl = I.workload("C5")
+    sweep(wl, 0, range(0, 2))

@@ -1,0 +1,154 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.  Scores within 2e-3 relative / 1e-5 absolute; index
+sets, rank rows, statistic integers and compacted rows exact (index sets up to
+the tolerance band around the k-th score)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import asl_oracle as O
+from paper_2601_07667_b200 import inputs as I
+
+from asl_check import StatReplay, check_layer, make_path, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_stack(wl, seed, layers=None):
+    path = make_path(wl)
+    replay = StatReplay(wl)
+    rels_gpu, rels_ref = [], []
+    for layer in (range(wl.layers) if layers is None else layers):
+        x = I.layer_inputs(wl, layer, seed)
+        res = check_layer(path, wl, x, layer)
+        recs = replay.step(path, layer, res)
+        iso, e2e = recs[0]
+        if iso["evaluated"]:
+            rels_gpu.append(iso["rel"])
+            rels_ref.append(e2e["rel"])
+    for b in range(wl.batch):
+        assert replay.on_gpu_scores[b].selected_layer == replay.on_ref_scores[b].selected_layer
+    if rels_gpu:
+        assert int(np.argmin(rels_gpu)) == int(np.argmin(rels_ref))
+    path.close()
+    return rels_gpu, rels_ref
+
+
+def test_c1_tiny_stack():
+    run_stack(I.workload("C1"), seed=0)
+
+
+def test_c1_other_seed_planted_keys_are_kept():
+    wl = I.workload("C1")
+    path = make_path(wl)
+    x = I.layer_inputs(wl, 0, seed=7)
+    check_layer(path, wl, x, 0)
+    idx = path.idx.cpu().numpy()
+    for h, pos in enumerate(I.planted_positions(wl, 7)[0]):
+        assert np.isin(pos, idx[h]).all()
+    path.close()
+
+
+@pytest.mark.parametrize("seqlens,budgets,w,S", [
+    ((33,), (32,), 32, 7),            # one past token, k = 0: window only
+    ((200,), (500,), 32, 7),          # budget >= n: keep everything
+    ((129,), (40,), 32, 1),           # S = 1, one key past a tile edge
+    ((1000, 257, 4097), (100, 257, 300), 16, 5),   # ragged batch, tile-edge lengths
+    ((700,), (96,), 24, 3),           # window that is not a power of two
+])
+def test_edge_shapes(seqlens, budgets, w, S):
+    wl = I.workload("C1", seqlens=seqlens, budgets=budgets, window=w, pool_kernel=S, layers=3, l_min=1, l_obs=2)
+    run_stack(wl, seed=3)
+
+
+def test_ragged_batch_small():
+    wl = I.workload("C4", seqlens=(3000, 5001, 2177, 4096), budgets=(300, 500, 217, 409), layers=3)
+    run_stack(wl, seed=1)
+
+
+def test_max_pool_wide_gqa_small():
+    wl = I.workload("C5", seqlens=(5000,), budgets=(600,), layers=4, l_min=1, l_obs=3)
+    run_stack(wl, seed=2)
+
+
+def test_topk_exact_ties_lowest_index_wins():
+    """Quantised scores: the k-th boundary falls inside long runs of exact ties."""
+    from paper_2601_07667_b200 import binding as B
+    wl = I.workload("C1", seqlens=(9000 + 32, 2500 + 32), budgets=(1500, 2500 + 32))
+    path = make_path(wl)
+    for levels in (3, 16, 200):
+        s = I.quantised_scores(wl.n_kv_heads, path.sum_T, levels, seed=levels)
+        path.scores_kv.copy_(torch.from_numpy(s))
+        B.asl_select_topk(path.ctx, path.scores_kv, wl.n_kv_heads, path.idx, path.workspace, path.ws_bytes)
+        torch.cuda.synchronize()
+        idx = path.idx.cpu().numpy()
+        for b in range(wl.batch):
+            n, w = wl.seqlens[b], wl.window
+            ts, ko, kept = int(path.t_off[b]), int(path.kept_off[b]), wl.kept(b)
+            for h in range(wl.n_kv_heads):
+                ref = O.select_topk(s[h, ts:ts + n - w].astype(np.float64), kept - w, n, w)
+                assert (idx[h, ko:ko + kept] == ref).all()
+    path.close()
+
+
+def test_rank_rows_with_ties_and_statistic_on_planted_rank_rows():
+    """asl_rank_stat alone: tied scores, and a ring whose statistic has a closed form."""
+    from paper_2601_07667_b200 import binding as B
+    T, w = 10000, 32
+    wl = I.workload("C1", seqlens=(T + w,), budgets=(T + w,), l_min=0, l_obs=2)       # k = T
+    path = make_path(wl)
+    asc = torch.arange(T, dtype=torch.float32, device="cuda")
+    for layer, agg in enumerate([asc, -asc]):                     # rank rows: reversed, identity
+        path.scores_agg.copy_(agg)
+        B.asl_rank_stat(path.ctx, path.scores_agg, layer, layer + 1, path.rank_ring, path.stat, path.workspace,
+                        path.ws_bytes)
+    torch.cuda.synchronize()
+    st = path.read_stat()[0]
+    assert st["evaluated"] == 1 and st["m"] == T and st["rows"] == 2
+    assert st["var_top"] == pytest.approx((T * T - 1) / 12.0, rel=1e-14)       # reversed ranks, k = T
+    assert st["rel"] == 1.0 and st["selected"] == 0
+    ties = torch.from_numpy(I.quantised_scores(1, T, 7, seed=9)[0]).cuda()
+    path.scores_agg.copy_(ties)
+    B.asl_rank_stat(path.ctx, path.scores_agg, 2, 2, path.rank_ring, path.stat, path.workspace, path.ws_bytes)
+    torch.cuda.synchronize()
+    assert (path.rank_ring[0].cpu().numpy() == O.rank_desc(ties.cpu().numpy().astype(np.float64))).all()
+    path.close()
+
+
+def test_invalid_arguments_are_refused():
+    from paper_2601_07667_b200 import binding as B
+    ctx = B.asl_create(0)
+    base = dict(n_q_heads=8, n_kv_heads=2, head_dim=128, window=32, pool_kernel=7, pool_mode=0,
+                cu_seqlens=[0, 100], budgets=[64], l_min=1, l_obs=2, tau=0.3,
+                q_stride=(8 * 32 * 128, 32 * 128, 128), k_stride=(256, 128), v_stride=(256, 128))
+    assert B.asl_plan(ctx, **base) > 0
+    for bad in (dict(pool_kernel=4), dict(cu_seqlens=[0, 32]), dict(budgets=[16]), dict(n_kv_heads=3),
+                dict(l_obs=1), dict(k_stride=(256, 127)), dict(window=0)):
+        with pytest.raises(B.AslError) as e:
+            B.asl_plan(ctx, **{**base, **bad})
+        assert e.value.status == B.ASL_ERR_INVALID
+    B.asl_plan(ctx, **base)
+    t = torch.zeros(1 << 20, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.AslError) as e:
+        B.asl_score_layer(ctx, t, t, t, t, t, 16)
+    assert e.value.status == B.ASL_ERR_WORKSPACE
+    with pytest.raises(B.AslError) as e:
+        B.asl_rank_stat(ctx, t, 0, 2, t, t, t, t.numel() * 4)            # n_rows > layer_idx + 1
+    assert e.value.status == B.ASL_ERR_INVALID
+    assert B.asl_device_status(ctx)[0] == B.ASL_OK
+    B.asl_destroy(ctx)
+
+
+def test_run_twice_is_bitwise_identical():
+    wl = I.workload("C1")
+    x = I.layer_inputs(wl, 1, seed=4)
+    q, k, v = to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])
+    outs = []
+    for _ in range(2):
+        path = make_path(wl)
+        path.run_layer(q, k, v, 0)
+        torch.cuda.synchronize()
+        outs.append((path.scores_kv.clone(), path.scores_agg.clone(), path.idx.clone(), path.rank_ring.clone()))
+        path.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
