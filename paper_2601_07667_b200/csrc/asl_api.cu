@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, planning, workspace layout, dispatch.
 #include <math.h>
+#include <stdlib.h>
 #include <new>
 
 #include "asl_internal.cuh"
@@ -9,6 +10,7 @@ namespace {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 void free_plan(asl_ctx* c) {
+  asl_tc_free(c);
   if (c->d_req) cudaFree(c->d_req);
   if (c->d_acc) cudaFree(c->d_acc);
   c->d_req = nullptr;
@@ -31,6 +33,8 @@ asl_status asl_create(asl_ctx** out, int device) {
   asl_ctx* c = new (std::nothrow) asl_ctx();
   if (!c) return ASL_ERR_CUDA;
   c->device = device;
+  const char* fs = getenv("ASL_FORCE_SIMT");
+  c->force_simt = fs && fs[0] == '1';
   c->sm_count = prop.multiProcessorCount;
   int prev = 0;
   cudaGetDevice(&prev);
@@ -120,11 +124,21 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   c->rows_per_kv = (p->n_q_heads / p->n_kv_heads) * p->window;
   c->n_key_tiles = (int32_t)tiles;
 
+  cudaGetDevice(&prev);
+  cudaSetDevice(c->device);
+  const bool tc = asl_tc_plan(c);
+  cudaSetDevice(prev);
+  const int G = p->n_q_heads / p->n_kv_heads;
+  c->u_rows_per_kv = p->pool_mode == ASL_POOL_MAX ? G : (tc ? c->tc.nchunk : 1);
+
   AslWorkspace& w = c->ws;
   size_t off = 0;
-  w.score_partials = off; off = asl_align256(off + (size_t)tiles * p->n_kv_heads * c->rows_per_kv * sizeof(float2));
+  size_t partial_bytes = (size_t)tiles * p->n_kv_heads * c->rows_per_kv * sizeof(float2);
+  if (tc && c->tc.units1.size() * c->tc.NC * sizeof(float2) > partial_bytes)
+    partial_bytes = c->tc.units1.size() * c->tc.NC * sizeof(float2);
+  w.score_partials = off; off = asl_align256(off + partial_bytes);
   w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * c->rows_per_kv * sizeof(float));
-  const size_t u_rows = p->pool_mode == ASL_POOL_MAX ? p->n_q_heads : p->n_kv_heads;
+  const size_t u_rows = (size_t)p->n_kv_heads * c->u_rows_per_kv;
   w.score_u = off;        off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float));
   w.score_end = off;
   for (int i = 0; i < 2; ++i) { w.rank_keys[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
@@ -152,6 +166,9 @@ asl_status asl_score_layer(asl_ctx* c, const void* q_obs, const void* k, float* 
   if (!c || !c->planned || !q_obs || !k || !scores_kv || !scores_agg) return ASL_ERR_INVALID;
   if (!aligned16(q_obs) || !aligned16(k)) return ASL_ERR_INVALID;
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  if (c->tc.enabled && !c->force_simt)
+    return asl_launch_score_tc(c, q_obs, k, scores_kv, scores_agg, static_cast<char*>(workspace),
+                               static_cast<cudaStream_t>(stream));
   return asl_launch_score_simt(c, q_obs, k, scores_kv, scores_agg, static_cast<char*>(workspace),
                                static_cast<cudaStream_t>(stream));
 }

@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "asl.h"
+#include "score_tc.cuh"
 
 // Per-request table entry, one per request, resident on the device.
 struct AslReq {
@@ -37,6 +38,7 @@ struct asl_ctx {
   int device = 0;
   int sm_count = 0;
   bool planned = false;
+  bool force_simt = false;            // set from ASL_FORCE_SIMT=1 at create time (debugging aid)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
   std::vector<AslReq> req;
@@ -48,7 +50,8 @@ struct asl_ctx {
   // scorer plan
   int32_t rows_per_kv = 0;            // G*W
   int32_t n_key_tiles = 0;            // sum over requests of ceil(n_b / tile)
-  int32_t p1_splits = 0;              // partials per row written by pass 1
+  int32_t u_rows_per_kv = 1;          // rows of un-pooled column sums per kv head (chunks, or G for max pooling)
+  AslTcPlan tc;                       // tensor-core scorer plan (enabled when the shape fits)
   AslWorkspace ws{};
   int64_t launches = 0;
 };
@@ -64,6 +67,10 @@ static inline size_t asl_align256(size_t x) { return (x + 255) & ~size_t(255); }
 // ---- kernels' host launchers (one per translation unit) ----
 asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
                                  char* ws, cudaStream_t st);
+bool asl_tc_plan(asl_ctx* c);
+void asl_tc_free(asl_ctx* c);
+asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
+                               char* ws, cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);

@@ -1,7 +1,8 @@
 // 1-D pooling, GQA group sum and all-head aggregate (Algorithm 1 lines 5-6 and
 // the "scores" sum of Section 4.1).  One thread per past token walks the kv
 // heads, so the aggregate needs no atomics and is bit-reproducible.
-//   average pooling: input is the group-summed column sums u[H_k][sum_T]
+//   average pooling: input is group-summed column sums, `urows` rows per kv head
+//                    (one per row chunk of the scorer) that are added first
 //                    (pooling is linear, so summing the group first is the same
 //                    up to rounding); zero padding, divisor always S.
 //   max pooling:     input is per query head u[H_q][sum_T]; each head is
@@ -12,7 +13,7 @@
 namespace {
 
 __global__ void __launch_bounds__(256) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
-                                                         int Hk, int G, int S, int mode, int64_t sum_T,
+                                                         int Hk, int G, int S, int mode, int urows, int64_t sum_T,
                                                          float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
   const int b = blockIdx.y;
   const AslReq rq = req[b];
@@ -25,9 +26,11 @@ __global__ void __launch_bounds__(256) pool_group_kernel(const float* __restrict
   for (int h = 0; h < Hk; ++h) {
     float p;
     if (mode == ASL_POOL_AVG) {
-      const float* row = u + (int64_t)h * sum_T + rq.t_off;
       float s = 0.f;
-      for (int i = lo; i <= hi; ++i) s += row[i];
+      for (int c = 0; c < urows; ++c) {
+        const float* row = u + (int64_t)(h * urows + c) * sum_T + rq.t_off;
+        for (int i = lo; i <= hi; ++i) s += row[i];
+      }
       p = s * inv;
     } else {
       p = 0.f;
@@ -50,7 +53,7 @@ asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* 
   const asl_params& p = c->p;
   dim3 grid((c->max_T + 255) / 256, p.batch);
   pool_group_kernel<<<grid, 256, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
-                                          p.pool_mode, c->sum_T, scores_kv, scores_agg);
+                                          p.pool_mode, c->u_rows_per_kv, c->sum_T, scores_kv, scores_agg);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

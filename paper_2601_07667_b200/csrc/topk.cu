@@ -1,17 +1,28 @@
 // Per-(request, head) top-k with the window appended (Algorithm 1 lines 7-8).
 //
-// Radix select on an order-preserving 32-bit image of the fp32 score: four
-// most-significant-digit passes (8 bits each) find the exact k-th largest key;
-// every token with a larger key is kept, and of the tokens that equal it the
-// lowest-indexed ones fill the remainder.  An ordered block scan then emits the
-// kept indices in ascending order, followed by T .. n-1.
+// Radix select on an order-preserving 32-bit image of the fp32 score, 11+11+10
+// bits from the top: the exact k-th largest key is found; every token with a
+// larger key is kept, and of the tokens equal to it the lowest-indexed fill the
+// remainder.  One thread-block cluster (up to 8 CTAs of 1024 threads) works on
+// one (request, head): each thread keeps 16 consecutive scores in registers,
+// CTAs histogram their slices in shared memory, read each other's histograms
+// through distributed shared memory and agree on the digit; an ordered scan
+// then emits the kept indices in ascending order, followed by T .. n-1.
+// Segments longer than cluster x 16384 are walked in rounds and re-read from L2.
+#include <cooperative_groups.h>
+
 #include "asl_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
 constexpr int THREADS = 1024;
-constexpr int PER_THREAD = 4;
-constexpr int CHUNK = THREADS * PER_THREAD;
+constexpr int PER_THREAD = 16;
+constexpr int SLICE = THREADS * PER_THREAD;   // scores per CTA per round
+constexpr int BINS = 2048;
+constexpr int MAX_CL = 8;
+constexpr int MAX_ROUNDS = 64;
 
 __device__ __forceinline__ uint32_t asc_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -19,106 +30,207 @@ __device__ __forceinline__ uint32_t asc_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(THREADS) topk_select_kernel(const float* __restrict__ scores,
-                                                              const AslReq* __restrict__ req, int64_t sum_T,
-                                                              int64_t sum_kept, int32_t* __restrict__ idx_out) {
-  __shared__ int hist[256];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_remaining;
-  __shared__ int warp_sums[THREADS / 32];
-  const int b = blockIdx.y, h = blockIdx.x;
+struct Shared {
+  int hist[BINS];
+  int tot[BINS];
+  int warp_a[32], warp_b[32];
+  int counts[MAX_ROUNDS][2];     // this CTA's (larger, equal) counts per round
+  uint32_t prefix;
+  int remaining;
+};
+
+template <bool CACHED>
+__global__ void __launch_bounds__(THREADS) topk_cluster_kernel(const float* __restrict__ scores,
+                                                               const AslReq* __restrict__ req, int64_t sum_T,
+                                                               int64_t sum_kept, int32_t* __restrict__ idx_out) {
+  __shared__ Shared sh;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int CL = (int)cluster.num_blocks();
+  const int r = (int)cluster.block_rank();
+  const int b = blockIdx.z, h = blockIdx.y;
   const AslReq rq = req[b];
   const float* row = scores + (int64_t)h * sum_T + rq.t_off;
   int32_t* out = idx_out + (int64_t)h * sum_kept + rq.kept_off;
   const int T = rq.T, k = rq.k;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int rounds = (T + CL * SLICE - 1) / (CL * SLICE);
 
   // window indices (Algorithm 1 line 8)
-  for (int t = tid; t < rq.kept - k; t += THREADS) out[k + t] = T + t;
-  if (k == 0) return;
+  for (int t = r * THREADS + tid; t < rq.kept - k; t += CL * THREADS) out[k + t] = T + t;
+  if (k == 0) return;                      // uniform over the cluster: nobody waits for anybody
 
-  // ---- exact k-th largest key -------------------------------------------------
-  uint32_t prefix = 0, mask = 0;
-  int remaining = k;     // rank of the wanted key among keys matching the prefix (1 = largest)
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
-    for (int i = tid; i < T; i += THREADS) {
-      const uint32_t u = asc_key(row[i]);
-      if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255], 1);
-    }
-    __syncthreads();
-    if (tid == 0) {
-      int rem = remaining, d = 255;
-      for (; d > 0; --d) {
-        if (hist[d] >= rem) break;
-        rem -= hist[d];
-      }
-      s_prefix = prefix | ((uint32_t)d << shift);
-      s_remaining = rem;
-    }
-    __syncthreads();
-    prefix = s_prefix;
-    remaining = s_remaining;
-    mask |= 0xFFu << shift;
-    __syncthreads();
-  }
-  const uint32_t thr = prefix;       // k-th largest key
-  const int need = remaining;        // how many keys equal to thr are kept (lowest indices)
-
-  // ---- ordered emit -------------------------------------------------------------
-  const int lane = tid & 31, wid = tid >> 5;
-  int run_gt = 0, run_eq = 0;        // kept-larger / equal counts before this chunk
-  for (int c0 = 0; c0 < T; c0 += CHUNK) {
-    const int i0 = c0 + tid * PER_THREAD;
-    uint32_t u[PER_THREAD];
-    int packed = 0;                  // (larger << 16) | equal, each <= 4096*... per chunk <= CHUNK < 65536
+  uint32_t key[PER_THREAD];
+  auto load_round = [&](int rho) {
+    const int i0 = (rho * CL + r) * SLICE + tid * PER_THREAD;
 #pragma unroll
-    for (int e = 0; e < PER_THREAD; ++e) {
-      const int i = i0 + e;
-      u[e] = (i < T) ? asc_key(row[i]) : 0u;
-      if (i < T) packed += (u[e] > thr) ? (1 << 16) : ((u[e] == thr) ? 1 : 0);
+    for (int e = 0; e < PER_THREAD; ++e) key[e] = (i0 + e < T) ? asc_key(__ldg(row + i0 + e)) : 0u;
+  };
+  if (CACHED) load_round(0);
+
+  // ---- exact k-th largest key: three digit passes ---------------------------------
+  uint32_t prefix = 0, mask = 0;
+  int remaining = k;
+  const int shifts[3] = {21, 10, 0};
+  const int widths[3] = {11, 11, 10};
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = shifts[pass];
+    const uint32_t dmask = (1u << widths[pass]) - 1u;
+    for (int i = tid; i < BINS; i += THREADS) sh.hist[i] = 0;
+    __syncthreads();
+    for (int rho = 0; rho < rounds; ++rho) {
+      if (!CACHED) load_round(rho);
+      const int i0 = (rho * CL + r) * SLICE + tid * PER_THREAD;
+#pragma unroll
+      for (int e = 0; e < PER_THREAD; ++e) {
+        const bool in = (i0 + e < T) && ((key[e] & mask) == prefix);
+        const int d = in ? (int)((key[e] >> shift) & dmask) : (BINS + lane);
+        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        if (in && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&sh.hist[d], __popc(peers));
+      }
     }
-    int incl = packed;
+    cluster.sync();                        // every CTA's histogram is complete
+    for (int i = tid; i < BINS; i += THREADS) {
+      int s = 0;
+      for (int c = 0; c < CL; ++c) s += cluster.map_shared_rank(sh.hist, c)[i];
+      sh.tot[i] = s;
+    }
+    cluster.sync();                        // remote reads done: histograms may be cleared again
+    // suffix sums from the top bin: thread t owns bins 2047-2t and 2046-2t
+    const int hi = BINS - 1 - 2 * tid, lo = hi - 1;
+    const int c_hi = sh.tot[hi], c_lo = sh.tot[lo];
+    int incl = c_hi + c_lo;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       int v = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += v;
     }
-    if (lane == 31) warp_sums[wid] = incl;
+    if (lane == 31) sh.warp_a[wid] = incl;
     __syncthreads();
-    int base = 0, total = 0;
-    for (int w2 = 0; w2 < THREADS / 32; ++w2) {
-      const int v = warp_sums[w2];
-      if (w2 < wid) base += v;
-      total += v;
+    int base = 0;
+    for (int w2 = 0; w2 < wid; ++w2) base += sh.warp_a[w2];
+    const int before_hi = base + incl - (c_hi + c_lo);     // keys in bins above `hi`
+    const int before_lo = before_hi + c_hi;
+    if (before_hi < remaining && remaining <= before_hi + c_hi) {
+      sh.prefix = prefix | ((uint32_t)hi << shift);
+      sh.remaining = remaining - before_hi;
+    } else if (before_lo < remaining && remaining <= before_lo + c_lo) {
+      sh.prefix = prefix | ((uint32_t)lo << shift);
+      sh.remaining = remaining - before_lo;
     }
-    int excl = base + incl - packed;
-    int gt_before = run_gt + (excl >> 16), eq_before = run_eq + (excl & 0xFFFF);
+    __syncthreads();
+    prefix = sh.prefix;
+    remaining = sh.remaining;
+    mask |= dmask << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = prefix;             // the k-th largest key
+  const int need = remaining;              // keys equal to thr that are kept (lowest indices first)
+
+  // ---- counts per (round, CTA), then the ordered emit -------------------------------
+  for (int rho = 0; rho < rounds; ++rho) {
+    if (!CACHED) load_round(rho);
+    const int i0 = (rho * CL + r) * SLICE + tid * PER_THREAD;
+    int gt = 0, eq = 0;
+#pragma unroll
+    for (int e = 0; e < PER_THREAD; ++e) {
+      if (i0 + e < T) { gt += key[e] > thr; eq += key[e] == thr; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      gt += __shfl_down_sync(0xffffffffu, gt, o);
+      eq += __shfl_down_sync(0xffffffffu, eq, o);
+    }
+    if (lane == 0) { sh.warp_a[wid] = gt; sh.warp_b[wid] = eq; }
+    __syncthreads();
+    if (tid == 0) {
+      int g = 0, q = 0;
+      for (int w2 = 0; w2 < 32; ++w2) { g += sh.warp_a[w2]; q += sh.warp_b[w2]; }
+      sh.counts[rho][0] = g;
+      sh.counts[rho][1] = q;
+    }
+    __syncthreads();
+  }
+  cluster.sync();                          // every CTA's counts are visible
+  int run_gt = 0, run_eq = 0;              // kept-larger / equal keys before this CTA's slice of round 0
+  for (int c = 0; c < r; ++c) {
+    const int(*rc)[2] = cluster.map_shared_rank(sh.counts, c);
+    run_gt += rc[0][0];
+    run_eq += rc[0][1];
+  }
+  for (int rho = 0; rho < rounds; ++rho) {
+    if (!CACHED) load_round(rho);
+    const int i0 = (rho * CL + r) * SLICE + tid * PER_THREAD;
+    int gt = 0, eq = 0;
+#pragma unroll
+    for (int e = 0; e < PER_THREAD; ++e) {
+      if (i0 + e < T) { gt += key[e] > thr; eq += key[e] == thr; }
+    }
+    int ig = gt, ie = eq;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int vg = __shfl_up_sync(0xffffffffu, ig, o), ve = __shfl_up_sync(0xffffffffu, ie, o);
+      if (lane >= o) { ig += vg; ie += ve; }
+    }
+    __syncthreads();
+    if (lane == 31) { sh.warp_a[wid] = ig; sh.warp_b[wid] = ie; }
+    __syncthreads();
+    int gt_before = run_gt + ig - gt, eq_before = run_eq + ie - eq;
+    for (int w2 = 0; w2 < wid; ++w2) { gt_before += sh.warp_a[w2]; eq_before += sh.warp_b[w2]; }
 #pragma unroll
     for (int e = 0; e < PER_THREAD; ++e) {
       const int i = i0 + e;
       if (i < T) {
-        if (u[e] > thr) {
+        if (key[e] > thr) {
           out[gt_before + min(eq_before, need)] = i;
           ++gt_before;
-        } else if (u[e] == thr) {
+        } else if (key[e] == thr) {
           if (eq_before < need) out[gt_before + eq_before] = i;
           ++eq_before;
         }
       }
     }
-    run_gt += total >> 16;
-    run_eq += total & 0xFFFF;
-    __syncthreads();
+    if (rho + 1 < rounds) {                // counts of the slices between this one and ours in the next round
+      for (int c = r; c < CL; ++c) {
+        const int(*rc)[2] = cluster.map_shared_rank(sh.counts, c);
+        run_gt += rc[rho][0];
+        run_eq += rc[rho][1];
+      }
+      for (int c = 0; c < r; ++c) {
+        const int(*rc)[2] = cluster.map_shared_rank(sh.counts, c);
+        run_gt += rc[rho + 1][0];
+        run_eq += rc[rho + 1][1];
+      }
+    }
   }
+  cluster.sync();                          // no CTA leaves while its shared memory may still be read
 }
 
 }  // namespace
 
 asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, cudaStream_t st) {
-  topk_select_kernel<<<dim3(n_heads, c->p.batch), THREADS, 0, st>>>(scores, c->d_req, c->sum_T, c->sum_kept, idx_out);
+  int cl = (c->max_T + SLICE - 1) / SLICE;
+  if (cl < 1) cl = 1;
+  if (cl > MAX_CL) cl = MAX_CL;
+  const int rounds = (c->max_T + cl * SLICE - 1) / (cl * SLICE);
+  if (rounds > MAX_ROUNDS) return ASL_ERR_UNSUPPORTED;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(cl, n_heads, c->p.batch);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cl;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const AslReq* req = c->d_req;
+  int64_t sum_T = c->sum_T, sum_kept = c->sum_kept;
+  cudaError_t e;
+  if (rounds == 1) e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<true>, scores, req, sum_T, sum_kept, idx_out);
+  else             e = cudaLaunchKernelEx(&cfg, topk_cluster_kernel<false>, scores, req, sum_T, sum_kept, idx_out);
   c->launches += 1;
-  ASL_CUDA(cudaGetLastError());
+  if (e != cudaSuccess) return ASL_ERR_CUDA;
   return ASL_OK;
 }

@@ -125,7 +125,7 @@ def workload(name: str, seed: int = 0, **override) -> Workload:
     elif name == "C2":  # 8B-shaped layer sweep
         wl = Workload("C2", 2, 32, 32, 8, 128, 64, 7, POOL_AVG, (32768,), (2048,), 10, 8, 0.3,
                       heavy_per_head=16, heavy_decay=0.97, chan_scale="lognormal", chan_sigma=0.5,
-                      rope_base=500000.0, salience_start=0.0, salience_step=0.11, fresh_scale=1.0)
+                      rope_base=500000.0, salience_start=0.04, salience_step=0.035)
     elif name == "C3":  # long-context single request
         wl = Workload("C3", 3, 12, 32, 8, 128, 64, 7, POOL_AVG, (131072,), (4096,), 2, 8, 0.3,
                       heavy_per_head=1, distractors=64, distractor_cos=0.9)

@@ -61,6 +61,21 @@ def test_edge_shapes(seqlens, budgets, w, S):
     run_stack(wl, seed=3)
 
 
+@pytest.mark.parametrize("Hq,Hk,w,mode,n", [
+    (32, 8, 64, 0, 3000),     # 256-row chunks, average pooling (the 8B-shaped layout)
+    (8, 2, 128, 0, 2500),     # two 256-row chunks per kv head, average pooling
+    (8, 2, 32, 1, 2000),      # max pooling, two query heads per column half
+    (16, 2, 64, 1, 2100),     # max pooling, two chunks per kv head
+    (4, 2, 256, 1, 1500),     # window as large as a chunk
+    (4, 4, 64, 0, 1111),      # no grouping: 64-row chunk
+    (6, 2, 32, 0, 1000),      # 96-row chunk
+])
+def test_scorer_shapes(Hq, Hk, w, mode, n):
+    wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, pool_mode=mode, seqlens=(n,), budgets=(w + 100,),
+                    layers=2, l_min=1, l_obs=2)
+    run_stack(wl, seed=5)
+
+
 def test_ragged_batch_small():
     wl = I.workload("C4", seqlens=(3000, 5001, 2177, 4096), budgets=(300, 500, 217, 409), layers=3)
     run_stack(wl, seed=1)
@@ -88,6 +103,23 @@ def test_topk_exact_ties_lowest_index_wins():
             for h in range(wl.n_kv_heads):
                 ref = O.select_topk(s[h, ts:ts + n - w].astype(np.float64), kept - w, n, w)
                 assert (idx[h, ko:ko + kept] == ref).all()
+    path.close()
+
+
+def test_topk_long_segment_walked_in_rounds():
+    """A segment longer than one cluster's register cache (8 x 16384 scores)."""
+    from paper_2601_07667_b200 import binding as B
+    T, w = 300000, 32
+    wl = I.workload("C1", seqlens=(T + w,), budgets=(5000,))
+    path = make_path(wl)
+    for levels in (5, 100000):
+        s = I.quantised_scores(wl.n_kv_heads, T, levels, seed=levels)
+        path.scores_kv.copy_(torch.from_numpy(s))
+        B.asl_select_topk(path.ctx, path.scores_kv, wl.n_kv_heads, path.idx, path.workspace, path.ws_bytes)
+        torch.cuda.synchronize()
+        idx = path.idx.cpu().numpy()
+        for h in range(wl.n_kv_heads):
+            assert (idx[h] == O.select_topk(s[h].astype(np.float64), 5000 - w, T + w, w)).all()
     path.close()
 
 
