@@ -161,11 +161,24 @@ def time_oracle(wl, layer_sets, steps, warmup, heads):
     return wl.total_tokens * frac / dt, dt
 
 
+def make_workload(args):
+    """The named workload, optionally with other context lengths (profiling-sized cases)."""
+    base = I.workload(args.workload, seed=args.seed)
+    if not args.seqlens and not args.budgets:
+        return base
+    seqlens = tuple(int(x) for x in args.seqlens.split(",")) if args.seqlens else base.seqlens
+    if args.budgets:
+        budgets = tuple(int(x) for x in args.budgets.split(","))
+    else:                                          # keep the workload's first budget, one per request
+        budgets = tuple(min(base.budgets[0], n) for n in seqlens)
+    return I.workload(args.workload, seed=args.seed, seqlens=seqlens, budgets=budgets)
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    wl = I.workload(args.workload, seed=args.seed)
+    wl = make_workload(args)
     heads = 1
     sets = [I.layer_inputs(wl, l, args.seed) for l in range(2)]
     np.dot(np.ones((64, 64)), np.ones((64, 64)))
@@ -197,7 +210,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    wl = I.workload(args.workload, seed=args.seed)
+    wl = make_workload(args)
     work = algorithmic_work(wl)
     pk = peaks()
 
@@ -387,6 +400,9 @@ def main():
     ap.add_argument("--layer-sets", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seqlens", type=str, default=None,
+                    help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
+    ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
