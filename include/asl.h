@@ -146,6 +146,39 @@ asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, i
 asl_status asl_compact_kv(asl_ctx* ctx, const void* k, const void* v, const int32_t* idx, void* k_out,
                           void* v_out, void* stream);
 
+/* Rank row without any allocation.  (The paper has no counterpart: this is a
+ * packaging of Algorithm 1 line 9 for hosts that may not allocate.)
+ *
+ * Who needs it: a caller that cannot obtain device memory at the time it wants
+ * a rank row -- an inference server whose memory pool was handed over to its
+ * own allocator at start-up, a plugin invoked inside another runtime's
+ * callback, a process run under a "no cudaMalloc after initialisation" rule.
+ * Such a caller can use neither asl_create/asl_plan (both allocate small device
+ * tables) nor a workspace it has nowhere to take from.  This call needs no
+ * context and no workspace: its sort scratch is a fixed array compiled into
+ * the library (about 4.1 MiB of device memory on every GPU that loads the
+ * library, held until the process exits).
+ *
+ *   scores    device fp32 [T]   one request's aggregate scores
+ *   rank_out  device int32 [T]  rank_out[j] = 0-based rank of token j by
+ *                               descending score, ties to the lower index --
+ *                               the same row asl_rank_stat writes into its ring
+ *   T         1 .. ASL_RANK_STATIC_MAX_T; larger -> ASL_ERR_WORKSPACE (the fixed
+ *             scratch is too small; use asl_rank_stat with a workspace instead)
+ *
+ * Runs on the calling thread's current device, asynchronously on `stream`;
+ * calls no cudaMalloc/cudaFree and no allocating library routine.  The first
+ * call on each device also looks up the scratch array's device address and
+ * checks the architecture (ASL_ERR_ARCH unless sm_100); make that first call
+ * outside any stream capture.  All calls on a device share the one scratch
+ * array, which keeps whatever the last call left in it (every call overwrites
+ * what it reads, nothing needs clearing): two calls whose kernels can overlap
+ * on the GPU -- different streams, no ordering between them -- race on it and
+ * give wrong ranks.  Issue them on one stream or order them with events.
+ * ASL_ERR_INVALID for null pointers or T < 1. */
+#define ASL_RANK_STATIC_MAX_T 262144
+asl_status asl_rank_desc_static(const float* scores, int32_t T, int32_t* rank_out, void* stream);
+
 /* Reads the device error word written by bounded waits (host-synchronising:
  * it waits for `stream` first).  ASL_OK, or ASL_ERR_TIMEOUT with *where set to
  * the code of the wait that gave up; the word is cleared. */

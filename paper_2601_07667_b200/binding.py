@@ -18,7 +18,9 @@ ASL_OK, ASL_ERR_INVALID, ASL_ERR_UNSUPPORTED, ASL_ERR_WORKSPACE = 0, -1, -2, -3
 ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
-           "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror")
+           "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
+           "asl_rank_desc_static")
+ASL_RANK_STATIC_MAX_T = 262144
 
 
 class AslParams(C.Structure):
@@ -64,6 +66,7 @@ def _load() -> C.CDLL:
     lib.asl_select_topk.argtypes = [vp, vp, i32, vp, vp, sz, vp]
     lib.asl_compact_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.asl_device_status.argtypes = [vp, vp, C.POINTER(i32)]
+    lib.asl_rank_desc_static.argtypes = [vp, i32, vp, vp]
     lib.asl_launch_count.argtypes = [vp]
     lib.asl_launch_count.restype = i64
     lib.asl_strerror.argtypes = [C.c_int]
@@ -168,6 +171,17 @@ def asl_device_status(ctx, stream=None):
 
 def asl_launch_count(ctx) -> int:
     return int(_lib.asl_launch_count(ctx))
+
+
+def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
+    """Rank row of one request's scores with no context, no workspace and no
+    allocation: for callers that may not allocate device memory when they need
+    it (a server whose pool is owned by its own allocator, code inside another
+    runtime's callback).  The sort scratch is a fixed array inside the library,
+    shared by every call on the device, so calls that could overlap on the GPU
+    must be ordered; T is limited to ASL_RANK_STATIC_MAX_T."""
+    _check(_lib.asl_rank_desc_static(_ptr(scores), int(T), _ptr(rank_out), _stream_handle(stream)),
+           "asl_rank_desc_static")
 
 
 # ---- a small holder of one plan's device buffers -------------------------------------

@@ -11,6 +11,8 @@
 // (the k smallest ranks of a row are exactly ranks 0..k-1).  The numerator
 // sum_j (rows*sum r^2 - (sum r)^2) is accumulated in 64-bit integers with
 // integer atomics, so it does not depend on the order of accumulation.
+#include <mutex>
+
 #include "asl_internal.cuh"
 
 namespace {
@@ -241,6 +243,105 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
   rank_stat_finalize<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, evaluate,
                                                          p.tau);
   c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Allocation-free rank row.
+//
+// Some hosts of this library are not allowed to allocate device memory while
+// they run: a serving engine that hands its whole memory pool to its own
+// allocator at start-up, a plugin called from inside another runtime's
+// execution callback, code running under a "no cudaMalloc after init" rule.
+// For them the sort's scratch (two ping-pong key arrays, two payload arrays,
+// the per-tile digit histograms and a one-entry request table) lives in this
+// file-scope device array.  Every device that loads the library carries these
+// bytes until the process exits, which is why the segment length is capped.
+//
+// In host code `g_rank_static` is only a handle: the device address is asked
+// for once per device with cudaGetSymbolAddress and that pointer is what the
+// kernels get.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int STATIC_MAX_T = ASL_RANK_STATIC_MAX_T;
+constexpr int STATIC_NBLK = (STATIC_MAX_T + TILE - 1) / TILE;
+constexpr int STATIC_MAX_DEVICES = 64;
+
+struct RankStaticScratch {
+  AslReq req;                       // the one request the kernels index with blockIdx.y = 0
+  uint32_t keys[2][STATIC_MAX_T];
+  int32_t idx[2][STATIC_MAX_T];
+  int32_t hist[256 * STATIC_NBLK];
+};
+
+static __device__ __align__(256) unsigned char g_rank_static[sizeof(RankStaticScratch)];
+
+// Writes the request record.  Nothing else in the scratch has to start from a
+// known value: the sort writes every key, payload and histogram entry before it
+// reads it, so what an earlier call left behind is never seen.
+__global__ void rank_static_begin(RankStaticScratch* s, int T) {
+  AslReq r;
+  r.n = T; r.T = T; r.k = 0; r.kept = 0; r.tok_off = 0; r.t_off = 0; r.kept_off = 0; r.pad = 0;
+  s->req = r;
+}
+
+struct RankStaticDevices {
+  RankStaticScratch* ptr[STATIC_MAX_DEVICES] = {};
+  asl_status status[STATIC_MAX_DEVICES] = {};
+  bool done[STATIC_MAX_DEVICES] = {};
+  std::mutex lock;
+};
+
+RankStaticDevices& rank_static_devices() {
+  static RankStaticDevices d;
+  return d;
+}
+
+// Once per device, with that device current: architecture check and the
+// device address of the scratch array.
+asl_status rank_static_setup(int device, RankStaticScratch** out) {
+  RankStaticDevices& d = rank_static_devices();
+  std::lock_guard<std::mutex> guard(d.lock);
+  if (!d.done[device]) {
+    asl_status st = ASL_OK;
+    int major = 0;
+    void* p = nullptr;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) st = ASL_ERR_CUDA;
+    else if (major != 10) st = ASL_ERR_ARCH;
+    else if (cudaGetSymbolAddress(&p, g_rank_static) != cudaSuccess || !p) st = ASL_ERR_CUDA;
+    d.ptr[device] = static_cast<RankStaticScratch*>(p);
+    d.status[device] = st;
+    d.done[device] = true;
+  }
+  *out = d.ptr[device];
+  return d.status[device];
+}
+
+}  // namespace
+
+extern "C" asl_status asl_rank_desc_static(const float* scores, int32_t T, int32_t* rank_out, void* stream) {
+  if (!scores || !rank_out || T < 1) return ASL_ERR_INVALID;
+  if (T > STATIC_MAX_T) return ASL_ERR_WORKSPACE;      // the fixed scratch cannot hold this segment
+  int device = -1;
+  ASL_CUDA(cudaGetDevice(&device));
+  if (device < 0 || device >= STATIC_MAX_DEVICES) return ASL_ERR_UNSUPPORTED;
+  RankStaticScratch* s = nullptr;
+  const asl_status ready = rank_static_setup(device, &s);
+  if (ready != ASL_OK) return ready;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const AslReq* req = &s->req;
+  const int nblk = (T + TILE - 1) / TILE;
+  rank_static_begin<<<1, 1, 0, st>>>(s, T);
+  rank_prepare<<<dim3((T + 255) / 256, 1), 256, 0, st>>>(scores, req, s->keys[0], s->idx[0]);
+  for (int pass = 0; pass < 4; ++pass) {
+    const int in = pass & 1, out = in ^ 1;
+    rank_hist<<<dim3(nblk, 1), SORT_THREADS, 0, st>>>(s->keys[in], req, pass * 8, nblk, s->hist);
+    rank_scan<<<1, 256, 0, st>>>(s->hist, nblk);
+    rank_scatter<<<dim3(nblk, 1), SORT_THREADS, 0, st>>>(s->keys[in], s->idx[in], s->keys[out], s->idx[out],
+                                                         pass == 3 ? rank_out : nullptr, s->hist, req, pass * 8, nblk);
+  }
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;
 }
