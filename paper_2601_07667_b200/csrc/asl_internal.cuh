@@ -79,4 +79,4 @@ asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const in
                               cudaStream_t st);
 
 constexpr int ASL_SIMT_KEY_TILE = 128;   // keys per block in the SIMT scorer
-constexpr int ASL_RANK_TILE = 4096;      // keys per block in the radix sort
+constexpr int ASL_RANK_TILE = 2048;      // keys per block in the radix sort

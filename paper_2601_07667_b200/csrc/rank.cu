@@ -17,10 +17,11 @@
 
 namespace {
 
-constexpr int TILE = ASL_RANK_TILE;
+constexpr int TILE = ASL_RANK_TILE;      // keys per block
 constexpr int SORT_THREADS = 256;
 constexpr int WARPS = SORT_THREADS / 32;
-constexpr int PER_WARP = TILE / WARPS;   // 512 keys, walked 32 at a time
+constexpr int PER_WARP = TILE / WARPS;   // consecutive keys of one warp
+constexpr int ROUNDS = PER_WARP / 32;    // walked 32 at a time, all loads issued up front
 
 __device__ __forceinline__ uint32_t desc_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -29,59 +30,120 @@ __device__ __forceinline__ uint32_t desc_key(float s) {
   return ~u;                                             // ascending as the score descends
 }
 
-__global__ void rank_prepare(const float* __restrict__ agg, const AslReq* __restrict__ req, uint32_t* __restrict__ keys,
-                             int32_t* __restrict__ idx) {
-  const AslReq rq = req[blockIdx.y];
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= rq.T) return;
-  keys[rq.t_off + j] = desc_key(agg[rq.t_off + j]);
-  idx[rq.t_off + j] = j;
+// Lanes of the warp whose 8-bit digit equals this lane's: eight ballots, no
+// data-dependent loop (the hardware match instruction walks distinct values).
+__device__ __forceinline__ uint32_t same_digit(uint32_t d, bool valid) {
+  uint32_t peers = __ballot_sync(0xffffffffu, valid);
+#pragma unroll
+  for (int bit = 0; bit < 8; ++bit) {
+    const uint32_t b = __ballot_sync(0xffffffffu, (d >> bit) & 1u);
+    peers &= ((d >> bit) & 1u) ? b : ~b;
+  }
+  return peers;
 }
 
-// hist[b][digit][blk]: digit counts of one tile
-__global__ void __launch_bounds__(SORT_THREADS) rank_hist(const uint32_t* __restrict__ keys, const AslReq* __restrict__ req,
-                                                          int shift, int nblk, int32_t* __restrict__ hist) {
+// The first pass reads the fp32 scores and forms keys on the fly (token index =
+// position); later passes read the (key, index) pairs of the previous pass.
+template <bool FIRST>
+__device__ __forceinline__ void load_tile(const float* __restrict__ agg, const uint32_t* __restrict__ keys_in,
+                                          const int32_t* __restrict__ idx_in, const AslReq& rq, int wstart, int lane,
+                                          uint32_t (&key)[ROUNDS], int32_t (&id)[ROUNDS]) {
+#pragma unroll
+  for (int r = 0; r < ROUNDS; ++r) {
+    const int i = wstart + r * 32 + lane;
+    key[r] = 0u;
+    id[r] = i;
+    if (i < rq.T) {
+      if (FIRST) key[r] = desc_key(agg[rq.t_off + i]);
+      else { key[r] = keys_in[rq.t_off + i]; id[r] = idx_in[rq.t_off + i]; }
+    }
+  }
+}
+
+// hist[b][blk][digit]: digit counts of one tile
+template <bool FIRST>
+__global__ void __launch_bounds__(SORT_THREADS) rank_hist(const float* __restrict__ agg, const uint32_t* __restrict__ keys,
+                                                          const AslReq* __restrict__ req, int shift, int nblk,
+                                                          int32_t* __restrict__ hist) {
   __shared__ int cnt[256];
   const int b = blockIdx.y, blk = blockIdx.x;
   const AslReq rq = req[b];
-  cnt[threadIdx.x] = 0;
-  __syncthreads();
   const int start = blk * TILE;
-  if (start < rq.T) {
-    const int end = min(rq.T, start + TILE);
-    for (int i = start + threadIdx.x; i < end; i += SORT_THREADS)
-      atomicAdd(&cnt[(keys[rq.t_off + i] >> shift) & 255], 1);
+  if (start >= rq.T) return;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  cnt[threadIdx.x] = 0;
+  uint32_t key[ROUNDS];
+  int32_t id[ROUNDS];
+  load_tile<FIRST>(agg, keys, nullptr, rq, start + wid * PER_WARP, lane, key, id);
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < ROUNDS; ++r) {
+    const bool valid = start + wid * PER_WARP + r * 32 + lane < rq.T;
+    const uint32_t d = (key[r] >> shift) & 255u;
+    const uint32_t peers = same_digit(d, valid);
+    if (valid && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&cnt[d], __popc(peers));
   }
   __syncthreads();
-  hist[((int64_t)b * 256 + threadIdx.x) * nblk + blk] = cnt[threadIdx.x];
+  hist[((int64_t)b * nblk + blk) * 256 + threadIdx.x] = cnt[threadIdx.x];
 }
 
-// exclusive scan of hist[b] in (digit, blk) order, in place
-__global__ void __launch_bounds__(256) rank_scan(int32_t* __restrict__ hist, int nblk) {
+// in place: hist[b][blk][digit] -> first output position of (digit, blk), i.e. the
+// exclusive scan in (digit, blk) order.  1024 threads: thread (part, digit) walks a
+// quarter of the tiles with its loads batched, the parts are chained through shared memory.
+__global__ void __launch_bounds__(1024) rank_scan(int32_t* __restrict__ hist, const AslReq* __restrict__ req, int nblk) {
+  __shared__ int part_tot[4][256];
   __shared__ int warp_tot[8];
-  int32_t* row = hist + ((int64_t)blockIdx.x * 256 + threadIdx.x) * nblk;
+  const int b = blockIdx.x;
+  const int used = (req[b].T + TILE - 1) / TILE;             // tiles of this request
+  const int d = threadIdx.x & 255, part = threadIdx.x >> 8;
+  const int per = (used + 3) / 4;
+  const int b0 = part * per, b1 = min(used, b0 + per);
+  int32_t* col = hist + (int64_t)b * nblk * 256 + d;
   int total = 0;
-  for (int i = 0; i < nblk; ++i) total += row[i];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  int incl = total;
+  for (int i0 = b0; i0 < b1; i0 += 8) {
+    int v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = (i0 + k < b1) ? col[(int64_t)(i0 + k) * 256] : 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) total += v[k];
+  }
+  part_tot[part][d] = total;
+  __syncthreads();
+  int digit_total = 0, before = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int t = part_tot[q][d];
+    digit_total += t;
+    if (q < part) before += t;
+  }
+  // exclusive scan of the digit totals over the 256 digits (every part computes it)
+  const int lane = threadIdx.x & 31, w8 = d >> 5;
+  int incl = digit_total;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int v = __shfl_up_sync(0xffffffffu, incl, o);
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += v;
   }
-  if (lane == 31) warp_tot[wid] = incl;
+  if (part == 0 && lane == 31) warp_tot[w8] = incl;
   __syncthreads();
-  int base = incl - total;
-  for (int w2 = 0; w2 < wid; ++w2) base += warp_tot[w2];
-  for (int i = 0; i < nblk; ++i) {
-    int v = row[i];
-    row[i] = base;
-    base += v;
+  int base = incl - digit_total + before;
+  for (int w2 = 0; w2 < w8; ++w2) base += warp_tot[w2];
+  for (int i0 = b0; i0 < b1; i0 += 8) {
+    int v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = (i0 + k < b1) ? col[(int64_t)(i0 + k) * 256] : 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (i0 + k < b1) col[(int64_t)(i0 + k) * 256] = base;
+      base += v[k];
+    }
   }
 }
 
 // stable scatter of one tile; on the last pass writes rank[token] = position
-__global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const uint32_t* __restrict__ keys_in,
+template <bool FIRST>
+__global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __restrict__ agg,
+                                                             const uint32_t* __restrict__ keys_in,
                                                              const int32_t* __restrict__ idx_in,
                                                              uint32_t* __restrict__ keys_out, int32_t* __restrict__ idx_out,
                                                              int32_t* __restrict__ rank_row, const int32_t* __restrict__ offs,
@@ -92,49 +154,72 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const uint32_t* __r
   const int start = blk * TILE;
   if (start >= rq.T) return;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&cnt[0][0])[i] = 0;
-  __syncthreads();
   const int wstart = start + wid * PER_WARP;
   const uint32_t lt = (1u << lane) - 1u;
-  // per-warp digit counts
-  for (int r = 0; r < PER_WARP / 32; ++r) {
-    const int i = wstart + r * 32 + lane;
-    const bool valid = i < rq.T;
-    const uint32_t key = valid ? keys_in[rq.t_off + i] : 0u;
-    const int d = valid ? (int)((key >> shift) & 255) : (256 + lane);
-    const uint32_t peers = __match_any_sync(0xffffffffu, d);
-    if (valid && (peers & lt) == 0) cnt[wid][d] += __popc(peers);
+  uint32_t key[ROUNDS];
+  int32_t id[ROUNDS];
+  load_tile<FIRST>(agg, keys_in, idx_in, rq, wstart, lane, key, id);
+  const int tile_off = offs[((int64_t)b * nblk + blk) * 256 + threadIdx.x];
+  for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&cnt[0][0])[i] = 0;
+  __syncthreads();
+  // per-warp digit counts; the peer masks are kept for the second walk
+  uint32_t peers[ROUNDS];
+#pragma unroll
+  for (int r = 0; r < ROUNDS; ++r) {
+    const bool valid = wstart + r * 32 + lane < rq.T;
+    const uint32_t d = (key[r] >> shift) & 255u;
+    peers[r] = same_digit(d, valid);
+    if (valid && (peers[r] & lt) == 0) cnt[wid][d] += __popc(peers[r]);
     __syncwarp();
   }
   __syncthreads();
   {  // digit threadIdx.x: bases of the warps, in warp order, after the tile's global offset
-    int run = offs[((int64_t)b * 256 + threadIdx.x) * nblk + blk];
+    int run = tile_off;
 #pragma unroll
     for (int w2 = 0; w2 < WARPS; ++w2) {
-      int v = cnt[w2][threadIdx.x];
+      const int v = cnt[w2][threadIdx.x];
       cnt[w2][threadIdx.x] = run;
       run += v;
     }
   }
   __syncthreads();
-  for (int r = 0; r < PER_WARP / 32; ++r) {
-    const int i = wstart + r * 32 + lane;
-    const bool valid = i < rq.T;
-    const uint32_t key = valid ? keys_in[rq.t_off + i] : 0u;
-    const int32_t id = valid ? idx_in[rq.t_off + i] : 0;
-    const int d = valid ? (int)((key >> shift) & 255) : (256 + lane);
-    const uint32_t peers = __match_any_sync(0xffffffffu, d);
+#pragma unroll
+  for (int r = 0; r < ROUNDS; ++r) {
+    const bool valid = wstart + r * 32 + lane < rq.T;
+    const uint32_t d = (key[r] >> shift) & 255u;
     int pos = 0;
-    if (valid) pos = cnt[wid][d] + __popc(peers & lt);
+    if (valid) pos = cnt[wid][d] + __popc(peers[r] & lt);
     __syncwarp();
-    if (valid && (peers & lt) == 0) cnt[wid][d] += __popc(peers);
+    if (valid && (peers[r] & lt) == 0) cnt[wid][d] += __popc(peers[r]);
     __syncwarp();
     if (valid) {
-      if (rank_row) rank_row[rq.t_off + id] = pos;
-      else { keys_out[rq.t_off + pos] = key; idx_out[rq.t_off + pos] = id; }
+      if (rank_row) rank_row[rq.t_off + id[r]] = pos;
+      else { keys_out[rq.t_off + pos] = key[r]; idx_out[rq.t_off + pos] = id[r]; }
     }
   }
 }
+
+// the four passes of one rank row; scratch: two key and two index arrays, tile histograms
+void launch_sort(const float* agg, const AslReq* req, int batch, int max_T, uint32_t* const keys[2], int32_t* const idx[2],
+                 int32_t* hist, int32_t* rank_row, cudaStream_t st) {
+  const int nblk = (max_T + TILE - 1) / TILE;
+  const dim3 grid(nblk, batch);
+  for (int pass = 0; pass < 4; ++pass) {
+    const int in = (pass + 1) & 1, out = in ^ 1;           // pass 0 reads the scores, writes buffer 0
+    const int shift = pass * 8;
+    int32_t* row = pass == 3 ? rank_row : nullptr;
+    if (pass == 0) {
+      rank_hist<true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, req, shift, nblk, hist);
+      rank_scan<<<batch, 1024, 0, st>>>(hist, req, nblk);
+      rank_scatter<true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, hist, req, shift, nblk);
+    } else {
+      rank_hist<false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], req, shift, nblk, hist);
+      rank_scan<<<batch, 1024, 0, st>>>(hist, req, nblk);
+      rank_scatter<false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, hist, req, shift, nblk);
+    }
+  }
+}
+
 
 struct StatArgs {
   const int32_t* ring;
@@ -221,19 +306,9 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
   int32_t* idx[2] = {reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[0]),
                      reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[1])};
   int32_t* hist = reinterpret_cast<int32_t*>(ws + c->ws.rank_hist);
-  const int nblk = (c->max_T + TILE - 1) / TILE;
   int32_t* row = ring + (int64_t)(layer_idx % p.l_obs) * c->sum_T;
-  rank_prepare<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(agg, c->d_req, keys[0], idx[0]);
-  c->launches += 1;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int in = pass & 1, out = in ^ 1;
-    const int shift = pass * 8;
-    rank_hist<<<dim3(nblk, p.batch), SORT_THREADS, 0, st>>>(keys[in], c->d_req, shift, nblk, hist);
-    rank_scan<<<p.batch, 256, 0, st>>>(hist, nblk);
-    rank_scatter<<<dim3(nblk, p.batch), SORT_THREADS, 0, st>>>(keys[in], idx[in], keys[out], idx[out],
-                                                               pass == 3 ? row : nullptr, hist, c->d_req, shift, nblk);
-    c->launches += 3;
-  }
+  launch_sort(agg, c->d_req, p.batch, c->max_T, keys, idx, hist, row, st);
+  c->launches += 12;
   const int evaluate = (layer_idx >= p.l_min && n_rows >= 2) ? 1 : 0;
   if (evaluate) {
     StatArgs a{ring, c->d_req, c->d_acc, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows};
@@ -332,16 +407,10 @@ extern "C" asl_status asl_rank_desc_static(const float* scores, int32_t T, int32
   if (ready != ASL_OK) return ready;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const AslReq* req = &s->req;
-  const int nblk = (T + TILE - 1) / TILE;
   rank_static_begin<<<1, 1, 0, st>>>(s, T);
-  rank_prepare<<<dim3((T + 255) / 256, 1), 256, 0, st>>>(scores, req, s->keys[0], s->idx[0]);
-  for (int pass = 0; pass < 4; ++pass) {
-    const int in = pass & 1, out = in ^ 1;
-    rank_hist<<<dim3(nblk, 1), SORT_THREADS, 0, st>>>(s->keys[in], req, pass * 8, nblk, s->hist);
-    rank_scan<<<1, 256, 0, st>>>(s->hist, nblk);
-    rank_scatter<<<dim3(nblk, 1), SORT_THREADS, 0, st>>>(s->keys[in], s->idx[in], s->keys[out], s->idx[out],
-                                                         pass == 3 ? rank_out : nullptr, s->hist, req, pass * 8, nblk);
-  }
+  uint32_t* const keys[2] = {s->keys[0], s->keys[1]};
+  int32_t* const idx[2] = {s->idx[0], s->idx[1]};
+  launch_sort(scores, req, 1, T, keys, idx, s->hist, rank_out, st);
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;
 }
