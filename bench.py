@@ -269,21 +269,8 @@ def run_ours(args):
     t_start.record(stream)
     for i in range(args.steps):
         s = dev_sets[(args.warmup + i) % n_sets]
-        a, b_ = ev(), ev()
-        a.record(stream)
-        B.asl_score_layer(path.ctx, s["q_obs"], s["k"], path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
-        b_.record(stream)
-        score_marks.append((a, b_))
-        li = args.warmup + i
-        rows = path.n_rows(li)
-        path._fork.record(stream)
-        path.side.wait_event(path._fork)
-        B.asl_rank_stat(path.ctx, path.scores_agg, li, rows, path.rank_ring, path.stat, path.workspace, path.ws_bytes,
-                        path.side)
-        path._join.record(path.side)
-        B.asl_select_topk(path.ctx, path.scores_kv, wl.n_kv_heads, path.idx, path.workspace, path.ws_bytes)
-        B.asl_compact_kv(path.ctx, s["k"], s["v"], path.idx, path.k_out, path.v_out)
-        stream.wait_event(path._join)
+        path.run_layer(s["q_obs"], s["k"], s["v"], args.warmup + i, score_marks=score_marks)
+    path.join()
     t_end.record(stream)
     barrier()
     launches = B.asl_launch_count(path.ctx) - launches0
@@ -322,6 +309,7 @@ def run_ours(args):
         idx_h.copy_(path.idx, non_blocking=True)
         ko_h.copy_(path.k_out, non_blocking=True)
         vo_h.copy_(path.v_out, non_blocking=True)
+        path.join()
         st_h.copy_(path.stat, non_blocking=True)
 
     path.reset()

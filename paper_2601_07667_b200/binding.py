@@ -189,7 +189,10 @@ class LayerPath:
     """Owns a context, its plan and the device buffers of one layer's pass
     (scores, indices, compacted cache, rank ring, statistic), all torch tensors.
     ``run_layer`` issues the five steps; the rank statistic goes to a side stream
-    so it overlaps the top-k and the compaction."""
+    and is not waited for: it overlaps the top-k and the compaction of its own
+    layer and the scoring of the next one (the aggregate scores are double
+    buffered for that).  ``join`` makes the current stream wait for it;
+    ``read_stat`` joins by itself.  A device-wide synchronize covers it too."""
 
     def __init__(self, *, n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, seqlens, budgets,
                  l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None):
@@ -217,7 +220,9 @@ class LayerPath:
         dev = self.dev
         self.workspace = torch.empty(max(self.ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.scores_kv = torch.empty((n_kv_heads, self.sum_T), dtype=torch.float32, device=dev)
-        self.scores_agg = torch.empty((self.sum_T,), dtype=torch.float32, device=dev)
+        self._agg = [torch.empty((self.sum_T,), dtype=torch.float32, device=dev) for _ in range(2)]
+        self._agg_free = [None, None]       # event after the statistic that last read the buffer
+        self._cur = 0
         self.idx = torch.empty((n_kv_heads, self.sum_kept), dtype=torch.int32, device=dev)
         self.k_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
         self.v_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
@@ -227,6 +232,15 @@ class LayerPath:
         self._fork = torch.cuda.Event()
         self._join = torch.cuda.Event()
         self.first_layer: Optional[int] = None
+
+    @property
+    def scores_agg(self):
+        """Aggregate scores of the latest layer (device fp32 [sum_T])."""
+        return self._agg[self._cur]
+
+    def join(self) -> None:
+        """The current stream waits for the statistic work issued so far."""
+        self.torch.cuda.current_stream().wait_event(self._join)
 
     def close(self) -> None:
         if self.ctx:
@@ -249,25 +263,39 @@ class LayerPath:
             self.first_layer = layer_idx
         return min(self.l_obs, layer_idx - self.first_layer + 1)
 
-    def run_layer(self, q_obs, k, v, layer_idx: int, *, overlap: bool = True) -> None:
-        """Steps a1..a5 for one layer on the current stream (statistic on the side stream)."""
+    def run_layer(self, q_obs, k, v, layer_idx: int, *, overlap: bool = True, score_marks=None) -> None:
+        """Steps a1..a5 for one layer on the current stream; with ``overlap`` the statistic
+        runs on the side stream and is left in flight (see ``join``).  ``score_marks``: a list
+        that receives a (start, end) event pair around the scoring call."""
         torch = self.torch
         ctx, ws, wsb = self.ctx, self.workspace, self.ws_bytes
         rows = self.n_rows(layer_idx)
-        asl_score_layer(ctx, q_obs, k, self.scores_kv, self.scores_agg, ws, wsb)
+        main = torch.cuda.current_stream()
+        self._cur ^= 1
+        agg = self._agg[self._cur]
+        if self._agg_free[self._cur] is not None:
+            main.wait_event(self._agg_free[self._cur])      # the statistic of two layers ago has read it
+        if score_marks is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(main)
+        asl_score_layer(ctx, q_obs, k, self.scores_kv, agg, ws, wsb)
+        if score_marks is not None:
+            e1.record(main)
+            score_marks.append((e0, e1))
         if overlap:
-            main = torch.cuda.current_stream()
             self._fork.record(main)
             self.side.wait_event(self._fork)
-            asl_rank_stat(ctx, self.scores_agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, self.side)
+            asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, self.side)
+            done = torch.cuda.Event()
+            done.record(self.side)
+            self._agg_free[self._cur] = done
             self._join.record(self.side)
         else:
-            asl_rank_stat(ctx, self.scores_agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb)
+            asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb)
         asl_select_topk(ctx, self.scores_kv, self.H_k, self.idx, ws, wsb)
         asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out)
-        if overlap:
-            torch.cuda.current_stream().wait_event(self._join)
 
     def read_stat(self) -> np.ndarray:
         """Device -> host copy of the [B] statistic records (synchronises)."""
+        self.join()
         return self.stat.cpu().numpy().view(STAT_DTYPE).reshape(self.batch)

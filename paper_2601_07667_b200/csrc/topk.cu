@@ -30,18 +30,6 @@ __device__ __forceinline__ uint32_t asc_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Lanes of the warp that are `in` and hold the same 11-bit digit as this lane: one
-// ballot per bit (the hardware match instruction walks the distinct values instead).
-__device__ __forceinline__ uint32_t same_bin(uint32_t d, bool in) {
-  uint32_t peers = __ballot_sync(0xffffffffu, in);
-#pragma unroll
-  for (int bit = 0; bit < 11; ++bit) {
-    const uint32_t b = __ballot_sync(0xffffffffu, (d >> bit) & 1u);
-    peers &= ((d >> bit) & 1u) ? b : ~b;
-  }
-  return peers;
-}
-
 struct Shared {
   int hist[BINS];
   int tot[BINS];
@@ -95,9 +83,7 @@ __global__ void __launch_bounds__(THREADS) topk_cluster_kernel(const float* __re
 #pragma unroll
       for (int e = 0; e < PER_THREAD; ++e) {
         const bool in = (i0 + e < T) && ((key[e] & mask) == prefix);
-        const uint32_t d = (key[e] >> shift) & dmask;
-        const uint32_t peers = same_bin(d, in);
-        if (in && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&sh.hist[d], __popc(peers));
+        if (in) atomicAdd(&sh.hist[(key[e] >> shift) & dmask], 1);     // shared-memory atomic: conflicts replay in hardware
       }
     }
     cluster.sync();                        // every CTA's histogram is complete
