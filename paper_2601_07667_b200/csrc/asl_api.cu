@@ -35,6 +35,8 @@ asl_status asl_create(asl_ctx** out, int device) {
   c->device = device;
   const char* fs = getenv("ASL_FORCE_SIMT");
   c->force_simt = fs && fs[0] == '1';
+  const char* sg = getenv("ASL_SCORE_GROUP");
+  c->score_group = sg ? atoi(sg) : 0;
   c->sm_count = prop.multiProcessorCount;
   int prev = 0;
   cudaGetDevice(&prev);
@@ -134,8 +136,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   AslWorkspace& w = c->ws;
   size_t off = 0;
   size_t partial_bytes = (size_t)tiles * p->n_kv_heads * c->rows_per_kv * sizeof(float2);
-  if (tc && c->tc.units1.size() * c->tc.NC * sizeof(float2) > partial_bytes)
-    partial_bytes = c->tc.units1.size() * c->tc.NC * sizeof(float2);
+  if (tc && asl_tc_partial_bytes(c) > partial_bytes) partial_bytes = asl_tc_partial_bytes(c);
   w.score_partials = off; off = asl_align256(off + partial_bytes);
   w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * c->rows_per_kv * sizeof(float));
   const size_t u_rows = (size_t)p->n_kv_heads * c->u_rows_per_kv;
@@ -205,6 +206,7 @@ asl_status asl_device_status(asl_ctx* c, void* stream, int32_t* where) {
   if (where) *where = word;
   if (word == 0) return ASL_OK;
   ASL_CUDA(cudaMemsetAsync(c->d_err, 0, sizeof(word), st));
+  if (asl_tc_reset_sync(c, st) != ASL_OK) return ASL_ERR_CUDA;
   return ASL_ERR_TIMEOUT;
 }
 

@@ -39,6 +39,7 @@ struct asl_ctx {
   int sm_count = 0;
   bool planned = false;
   bool force_simt = false;            // set from ASL_FORCE_SIMT=1 at create time (debugging aid)
+  int score_group = 0;                // set from ASL_SCORE_GROUP at create time (0: default phase grouping)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
   std::vector<AslReq> req;
@@ -69,6 +70,8 @@ asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float
                                  char* ws, cudaStream_t st);
 bool asl_tc_plan(asl_ctx* c);
 void asl_tc_free(asl_ctx* c);
+size_t asl_tc_partial_bytes(const asl_ctx* c);
+asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st);
 asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
                                char* ws, cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);

@@ -1,30 +1,40 @@
 // Observation-window scorer on the 5th-generation tensor cores (Algorithm 1 lines 3-4).
 //
-// One persistent CTA per SM streams 128-key tiles of bf16 K through a 4-stage
-// TMA ring into 128B-swizzled shared memory; one thread issues tcgen05.mma with
-// fp32 accumulators in tensor memory (two 256-column buffers, so the MMAs of
-// tile i+1 overlap the exponentials of tile i); eight warps read the
-// accumulators back with tcgen05.ld and do the softmax arithmetic in the log2
-// domain x = (q.k) * log2(e)/sqrt(d).
+// One persistent kernel, one CTA per SM, does both softmax passes of every
+// (request, kv head, row chunk) "segment":
 //
 //   pass 1  D[row][key] = Q_chunk . K_tile^T  (query rows in TMEM lanes): each
-//           thread owns one query row and keeps an online (max, sum); one
-//           partial per (work unit, row); a combine kernel folds a row's
-//           partials in unit order into offset = max + log2(sum).
+//           epilogue thread keeps, for its rows, the sum of 2^(x - ref) over the
+//           keys of the CTA's tiles (ref: the maximum of the first 32 keys the
+//           row met); each epilogue set publishes (ref, sum) per row.  Once every
+//           set has published, two helper warps per CTA fold the partials of
+//           "their" rows (row r belongs to CTA r mod grid), in a fixed order, into
+//           offset[row] = log2 of the row's softmax denominator, off the
+//           epilogue's critical path.
 //   pass 2  D[key][row] = K_tile . Q_chunk^T  (keys in TMEM lanes): each thread
 //           owns one key and sums exp2(x - offset[row]) over the chunk's rows:
 //           the key's column sum U, already summed over the GQA group.
 //
-// A "chunk" is up to 256 of the G*W query rows that share a kv head (the MMA's
-// N in pass 2); a "work unit" is a run of consecutive key tiles of one
-// (request, kv head, chunk).  Units are dealt round-robin to the CTAs in
-// (request, head, chunk, tile) order, so all CTAs work on the same kv head at
-// the same time.
+// All arithmetic is in the log2 domain x = (q.k) * log2(e)/sqrt(d).  A "chunk"
+// is up to 256 of the G*W query rows that share a kv head; a "phase" is one pass
+// over one segment's 128-key tiles.  Phases are ordered pass1(s0) pass1(s1)
+// pass2(s0) pass2(s1) pass1(s2) ... so that the offsets a pass-2 phase needs were
+// finished one phase earlier, and so that K of a segment is still in L2 when
+// pass 2 reads it again: HBM sees K once.  The tiles of the whole phase list are
+// dealt round-robin to the CTAs.
 //
-// Every wait on an mbarrier is bounded: when the limit is reached the thread
-// records a code in the context's error word, raises the CTA's abort flag and
-// all roles fall through to the common teardown (in-flight copies are waited
-// for with the same bound, tensor memory is freed).
+// Inside a CTA: warp 0 streams K tiles through a 3-stage TMA ring (128B-swizzled)
+// and keeps the Q chunks of two phases resident (the next one is prefetched);
+// warp 1 issues tcgen05.mma into two 256-column TMEM accumulators; warps 2-3 fold
+// pass-1 partials; two sets of four epilogue warps take alternate tiles, one
+// accumulator each, reading it with software-pipelined tcgen05.ld.  The
+// exponentials are split between the MUFU unit and a degree-3 polynomial on the
+// FMA pipe (packed f32x2 arithmetic).
+//
+// Every wait (mbarrier, counter) is bounded: when the limit is reached the thread
+// records a code in the context's error word and the CTA drains: producers stop,
+// the epilogue keeps walking its barrier sequence without waiting or computing,
+// in-flight copies are waited for with the same bound and tensor memory is freed.
 #include <cuda.h>
 
 #include "asl_internal.cuh"
@@ -32,26 +42,26 @@
 namespace {
 
 constexpr int KT = ASL_TC_KEY_TILE;          // keys per tile
-constexpr int NSTAGE = 4;
+constexpr int NSTAGE = 3;
 constexpr int HALF_BYTES = KT * 128;         // one 64-channel block of a K tile: 128 rows x 128 B
 constexpr int STAGE_BYTES = 2 * HALF_BYTES;
 constexpr int MAX_NC = 256;
-constexpr int Q_BLOCK_BYTES = MAX_NC * 128;  // one 64-channel block of the Q chunk
-constexpr int THREADS = 320;                 // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+constexpr int Q_BLOCK_BYTES = MAX_NC * 128;  // one 64-channel block of a Q chunk
+constexpr int Q_BUF_BYTES = 2 * Q_BLOCK_BYTES;
+constexpr int THREADS = 384;                 // warp 0: TMA, 1: MMA, 2-3: partial folding, 4-7 / 8-11: epilogue sets
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // every wait gives up after 2 s
 
-// shared-memory map (offsets from a 1024-aligned base)
-constexpr int SM_Q = 0;
-constexpr int SM_K = SM_Q + 2 * Q_BLOCK_BYTES;
-constexpr int SM_NEGOFF = SM_K + NSTAGE * STAGE_BYTES;       // float[256]
-constexpr int SM_SCRATCH = SM_NEGOFF + 1024;                 // float2[2][2][128] = 4 KB
-constexpr int SM_BAR = SM_SCRATCH + 4096;                    // mbarriers
+// shared-memory map (offsets from the 1024-aligned base of dynamic shared memory)
+constexpr int SM_Q = 0;                                      // two Q chunk buffers
+constexpr int SM_K = SM_Q + 2 * Q_BUF_BYTES;
+constexpr int SM_NEGOFF = SM_K + NSTAGE * STAGE_BYTES;       // float[2][256]: -offset per epilogue set
+constexpr int SM_BAR = SM_NEGOFF + 2048;                     // mbarriers
 constexpr int SM_MISC = SM_BAR + 128;                        // tmem base, abort flag
-constexpr int SM_TOTAL = SM_MISC + 64;
-constexpr int SMEM_BYTES = SM_TOTAL + 1024;                  // slack for the alignment
+constexpr int SMEM_BYTES = SM_MISC + 64;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget of one CTA");
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_TFULL = 2 * NSTAGE, BAR_TEMPTY = 2 * NSTAGE + 2,
-       BAR_QFULL = 2 * NSTAGE + 4, BAR_QEMPTY = 2 * NSTAGE + 5, BAR_DRAIN = 2 * NSTAGE + 6, N_BARS = 2 * NSTAGE + 7 };
+       BAR_QFULL = 2 * NSTAGE + 4, BAR_QEMPTY = 2 * NSTAGE + 6, BAR_DRAIN = 2 * NSTAGE + 8, N_BARS = 2 * NSTAGE + 9 };
 static_assert(N_BARS * 8 <= 128, "barrier area");
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -77,6 +87,11 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long now;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+  return now;
+}
 // Bounded wait.  `watch_abort`: also give up when another role raised the flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code,
                                           bool watch_abort) {
@@ -85,14 +100,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return true;
     if ((it & 15u) == 15u) {
       if (watch_abort && *abort_flag) return false;
-      unsigned long long now;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
       else if (now - t0 > WAIT_LIMIT_NS) break;
     }
   }
   *abort_flag = code;
   return false;
+}
+// Bounded wait until the 32-bit word at p equals `want` (acquire).  Lane 0 polls.
+__device__ __forceinline__ bool word_wait(const uint32_t* p, uint32_t want, volatile int* abort_flag, int code, int lane,
+                                          uint32_t nap_max) {
+  int gave_up = 0;
+  if (lane == 0) {
+    unsigned long long t0 = 0;
+    uint32_t nap = 64;
+    for (uint32_t it = 0;; ++it) {
+      uint32_t v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+      if (v == want) break;
+      if ((it & 7u) == 7u) {
+        const unsigned long long now = global_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > WAIT_LIMIT_NS || *abort_flag) { gave_up = 1; if (!*abort_flag) *abort_flag = code; break; }
+      }
+      __nanosleep(nap);
+      if (nap < nap_max) nap <<= 1;
+    }
+  }
+  return __shfl_sync(0xffffffffu, gave_up, 0) == 0;
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
@@ -125,9 +161,9 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum)
       : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 consecutive fp32 columns of this thread's TMEM lane: issue only; the
+// registers hold the data after tc_ld_wait on the same array.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -138,16 +174,101 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Waits for every tcgen05.ld this thread has issued.  The array is an in/out
+// operand so that no use of its registers can be scheduled above the wait.
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// ---- two fp32 values in one 64-bit register: the FMA pipe takes fma on such pairs as
+//      one instruction, which halves the issue slots of the softmax arithmetic ----
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ f32x2 pku(uint32_t lo, uint32_t hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void upku(f32x2 v, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ float hsum(f32x2 v) {
+  float lo, hi;
+  upk(v, lo, hi);
+  return lo + hi;
+}
+// 2^x of a pair on the MUFU unit
+__device__ __forceinline__ f32x2 ex2_pair_mufu(f32x2 x) {
+  float a, b;
+  upk(x, a, b);
+  return pk(ex2(a), ex2(b));
+}
+// 2^x of a pair on the FMA pipe (any x < 128): clamp at -125, round to the nearest
+// integer n with the 1.5*2^23 trick, degree-3 minimax polynomial of 2^f on
+// f = x - n in [-0.5, 0.5] (relative error 7.5e-5), n added into the exponent field.
+// Additions are written as fma(a, 1, b): the packed fma issues faster than the packed add.
+__device__ __forceinline__ f32x2 ex2_pair_poly(f32x2 x) {
+  float a, b;
+  upk(x, a, b);
+  const f32x2 xc = pk(fmaxf(a, -125.0f), fmaxf(b, -125.0f));
+  const f32x2 one = pk(1.0f, 1.0f);
+  const f32x2 t = fma2(xc, one, pk(12582912.0f, 12582912.0f));
+  const f32x2 f = fma2(fma2(t, one, pk(-12582912.0f, -12582912.0f)), pk(-1.0f, -1.0f), xc);
+  f32x2 p = fma2(pk(0.0551716685f, 0.0551716685f), f, pk(0.2426111400f, 0.2426111400f));
+  p = fma2(p, f, pk(0.6932609677f, 0.6932609677f));
+  p = fma2(p, f, pk(0.9999280572f, 0.9999280572f));
+  uint32_t tl, th, pl, ph;
+  upku(t, tl, th);
+  upku(p, pl, ph);
+  return pku(pl + (tl << 23), ph + (th << 23));
+}
+// which of a block's 16 column pairs take the polynomial: POLY_PAIRS_OF_8 of every 8, spread out
+#ifndef ASL_POLY_PAIRS_OF_8
+#define ASL_POLY_PAIRS_OF_8 2
+#endif
+constexpr int POLY_PAIRS_OF_8 = ASL_POLY_PAIRS_OF_8;
+__device__ __forceinline__ constexpr bool pair_is_poly(int pi) {
+  return POLY_PAIRS_OF_8 >= 4 ? (pi & 1) == 1
+                              : ((POLY_PAIRS_OF_8 >= 1 && (pi & 7) == 1) || (POLY_PAIRS_OF_8 >= 2 && (pi & 7) == 5) ||
+                                 (POLY_PAIRS_OF_8 >= 3 && (pi & 7) == 3));
+}
+// sum over 32 accumulator columns of 2^(v*scale + c), c one pair per column pair
+template <typename OffsetPair>
+__device__ __forceinline__ float exp_sum32(const uint32_t (&cur)[32], f32x2 scale2, OffsetPair off) {
+  f32x2 acc_m = pk(0.f, 0.f), acc_p = pk(0.f, 0.f);
+  const f32x2 one = pk(1.0f, 1.0f);
+#pragma unroll
+  for (int pi = 0; pi < 16; ++pi) {
+    const f32x2 x = fma2(pku(cur[2 * pi], cur[2 * pi + 1]), scale2, off(pi));
+    if (pair_is_poly(pi)) acc_p = fma2(ex2_pair_poly(x), one, acc_p);
+    else                  acc_m = fma2(ex2_pair_mufu(x), one, acc_m);
+  }
+  return hsum(fma2(acc_m, one, acc_p));
+}
 
 // K-major, 128B-swizzled operand: rows of 128 B, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -160,39 +281,64 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
 }
 
 struct TcArgs {
-  const TcUnit* units;
+  const TcPhase* phases;
   const AslReq* req;
-  float2* partials;        // pass 1 out: [unit][NC]
-  const float* offsets;    // pass 2 in:  [B][H_k][R]
+  float2* partials;        // pass 1: [segment][CTA][set][NC] (reference, sum) of each epilogue set
+  float* offsets;          // [segment][NC], written by the folding warps, read by pass 2
   float* u;                // pass 2 out: column sums
+  uint32_t* published;     // [segment] epilogue sets that have published, accumulated over launches
+  uint32_t* folded;        // [segment] rows whose offset is written, accumulated over launches
   int32_t* err;
   int64_t sum_T;
-  int32_t n_units, NC, W, G, Hk, R, u_rows_per_kv;
+  uint32_t epoch;          // launch number, from 1
+  int32_t n_phases, total_items, NC, W, G, Hk, u_rows_per_kv;
   float scale_log2;
 };
 
-template <int PASS, bool PER_Q>
+// walks the CTA's items (global item g = blockIdx.x + i*gridDim.x) through the phase list;
+// the current phase record stays in registers and is re-read only when g leaves it
+struct ItemWalk {
+  const TcPhase* phases;
+  int total;
+  int g, ph;
+  TcPhase cur;
+  __device__ __forceinline__ ItemWalk(const TcArgs& a) : phases(a.phases), total(a.total_items), g((int)blockIdx.x), ph(0) {
+    cur = phases[0];
+  }
+  __device__ __forceinline__ bool valid() const { return g < total; }
+  __device__ __forceinline__ const TcPhase& phase() {       // phases are sorted by g0 and cover [0, total)
+    while (g >= cur.g0 + cur.ntiles) cur = phases[++ph];
+    return cur;
+  }
+  __device__ __forceinline__ bool last_in_phase() const { return g + (int)gridDim.x >= cur.g0 + cur.ntiles; }
+  __device__ __forceinline__ void next() { g += (int)gridDim.x; }
+};
+
+template <bool PER_Q>
 __global__ void __launch_bounds__(THREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const TcArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {                       // the swizzled operand layout needs a 1024-byte aligned base
+    if (threadIdx.x == 0) atomicCAS(a.err, 0, 901);
+    return;
+  }
   const uint32_t bars = sbase + SM_BAR;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM_MISC + 4);
   float* s_negoff = reinterpret_cast<float*>(smem + SM_NEGOFF);
-  float2* s_scratch = reinterpret_cast<float2*>(smem + SM_SCRATCH);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = a.NC;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
-  // ---- set-up: zero the Q area (rows past NC feed unused MMA rows), barriers, tensor memory ----
-  for (int i = threadIdx.x; i < 2 * Q_BLOCK_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
+  // ---- set-up: zero the Q buffers (rows past NC feed unused MMA rows), barriers, tensor memory ----
+  for (int i = threadIdx.x; i < 2 * Q_BUF_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(BAR_FULL + s), 1); mbar_init(bar(BAR_EMPTY + s), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_TFULL + i), 1); mbar_init(bar(BAR_TEMPTY + i), 8); }
-    mbar_init(bar(BAR_QFULL), 1);
-    mbar_init(bar(BAR_QEMPTY), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_TFULL + i), 1); mbar_init(bar(BAR_TEMPTY + i), 4);
+      mbar_init(bar(BAR_QFULL + i), 1); mbar_init(bar(BAR_QEMPTY + i), 1);
+    }
     mbar_init(bar(BAR_DRAIN), 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,225 +355,342 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (warp == 0) {
     // =============================== TMA producer ===============================
+    // Local phase l (the l-th phase in which this CTA has a tile) uses Q buffer l%2.
     if (lane == 0) {
-      int tile_iter = 0, seg_iter = 0, cur_seg = -1;
+      ItemWalk w(a);
+      int item = 0, lp = -1, cur_ph = -1;
+      int q_issued = -1;                       // highest local phase whose Q chunk has been requested
+      int loaded_seg[2] = {-1, -1};
+      int next_ph = -1;                        // the CTA's next phase after the current one (-1: none)
+      int tok_off = 0;                         // first token of the current phase's request
       bool ok = true;
-      for (int ui = blockIdx.x; ok && ui < a.n_units; ui += gridDim.x) {
-        const TcUnit u = a.units[ui];
-        if (u.seg != cur_seg) {
-          if (seg_iter > 0 && !mbar_wait(bar(BAR_QEMPTY), (seg_iter - 1) & 1, s_abort, 11, true)) { ok = false; break; }
-          const int r0 = u.chunk * NC;
-          const int head = u.h * a.G + r0 / a.W, t0 = r0 % a.W;
-          mbar_expect_tx(bar(BAR_QFULL), 2u * 128u * (uint32_t)NC);
-          tma_load_4d(sbase + SM_Q, &tm_q, bar(BAR_QFULL), 0, t0, head, u.b);
-          tma_load_4d(sbase + SM_Q + Q_BLOCK_BYTES, &tm_q, bar(BAR_QFULL), 64, t0, head, u.b);
-          cur_seg = u.seg;
-          ++seg_iter;
+      // requests the Q chunk of local phase `l` (phase record p); `block`: wait for the buffer, else only try
+      auto issue_q = [&](int l, const TcPhase& p, bool block) -> bool {
+        const int b = l & 1, use = l >> 1;
+        if (use >= 1) {
+          const uint32_t par = (uint32_t)((use - 1) & 1);
+          if (block) { if (!mbar_wait(bar(BAR_QEMPTY + b), par, s_abort, 11, true)) return false; }
+          else if (!mbar_try(bar(BAR_QEMPTY + b), par)) return true;
         }
-        const int tok0 = a.req[u.b].tok_off + u.tile0 * KT;
-        for (int t = 0; t < u.ntiles; ++t, ++tile_iter) {
-          const int s = tile_iter % NSTAGE;
-          if (!mbar_wait(bar(BAR_EMPTY + s), ((tile_iter / NSTAGE) & 1) ^ 1, s_abort, 12, true)) { ok = false; break; }
-          mbar_expect_tx(bar(BAR_FULL + s), STAGE_BYTES);
-          const uint32_t dst = sbase + SM_K + s * STAGE_BYTES;
-          tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, u.h, tok0 + t * KT);
-          tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, u.h, tok0 + t * KT);
+        if (loaded_seg[b] == p.seg) {
+          mbar_arrive(bar(BAR_QFULL + b));     // same chunk as the buffer holds: nothing to copy
+        } else {
+          const int r0 = p.chunk * NC;
+          const int head = p.h * a.G + r0 / a.W, t0 = r0 % a.W;
+          const uint32_t dst = sbase + SM_Q + (uint32_t)b * Q_BUF_BYTES;
+          mbar_expect_tx(bar(BAR_QFULL + b), 2u * 128u * (uint32_t)NC);
+          tma_load_4d(dst, &tm_q, bar(BAR_QFULL + b), 0, t0, head, p.b);
+          tma_load_4d(dst + Q_BLOCK_BYTES, &tm_q, bar(BAR_QFULL + b), 64, t0, head, p.b);
+          loaded_seg[b] = p.seg;
         }
+        q_issued = l;
+        return true;
+      };
+      for (; ok && w.valid(); w.next(), ++item) {
+        const TcPhase p = w.phase();
+        if (w.ph != cur_ph) {
+          cur_ph = w.ph;
+          ++lp;
+          tok_off = a.req[p.b].tok_off;
+          if (q_issued < lp && !issue_q(lp, p, true)) { ok = false; break; }
+          // where does this CTA go after this phase?
+          const int end = p.g0 + p.ntiles;
+          const int gn = w.g + ((end - w.g + (int)gridDim.x - 1) / (int)gridDim.x) * (int)gridDim.x;
+          next_ph = -1;
+          if (gn < a.total_items) {
+            int q = w.ph + 1;
+            while (gn >= a.phases[q].g0 + a.phases[q].ntiles) ++q;
+            next_ph = q;
+          }
+        }
+        if (next_ph >= 0 && q_issued == lp) {    // prefetch the next phase's Q chunk once its buffer is free
+          if (!issue_q(lp + 1, a.phases[next_ph], false)) { ok = false; break; }
+        }
+        const int s = item % NSTAGE;
+        if (!mbar_wait(bar(BAR_EMPTY + s), ((item / NSTAGE) & 1) ^ 1, s_abort, 12, true)) { ok = false; break; }
+        mbar_expect_tx(bar(BAR_FULL + s), STAGE_BYTES);
+        const uint32_t dst = sbase + SM_K + s * STAGE_BYTES;
+        const int tok = tok_off + (w.g - p.g0) * KT;
+        tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok);
+        tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok);
       }
       if (!ok) {
         // let the copies already issued land before the CTA's shared memory is released
-        const int armed = tile_iter < NSTAGE ? tile_iter : NSTAGE;
+        const int armed = item < NSTAGE ? item : NSTAGE;
         for (int i = 0; i < armed; ++i) {
-          const int it = tile_iter - 1 - i, s = it % NSTAGE;
+          const int it = item - 1 - i, s = it % NSTAGE;
           mbar_wait(bar(BAR_FULL + s), (it / NSTAGE) & 1, s_abort, 13, false);
         }
+        for (int l = q_issued; l >= 0 && l > q_issued - 2; --l)
+          mbar_wait(bar(BAR_QFULL + (l & 1)), (l >> 1) & 1, s_abort, 14, false);
       }
     }
   } else if (warp == 1) {
     // =============================== MMA issuer =================================
     if (lane == 0) {
-      int tile_iter = 0, seg_iter = 0, cur_seg = -1;
+      ItemWalk w(a);
+      int item = 0, lp = -1, cur_ph = -1;
       bool ok = true;
-      const uint32_t idesc = (PASS == 1) ? instr_desc(128, KT) : instr_desc(KT, NC);
+      const uint32_t idesc1 = instr_desc(128, KT), idesc2 = instr_desc(KT, NC);
       const int nhalf = (NC > 128) ? 2 : 1;
-      for (int ui = blockIdx.x; ok && ui < a.n_units; ui += gridDim.x) {
-        const TcUnit u = a.units[ui];
-        if (u.seg != cur_seg) {
-          if (!mbar_wait(bar(BAR_QFULL), seg_iter & 1, s_abort, 21, true)) { ok = false; break; }
-          cur_seg = u.seg;
-          ++seg_iter;
+      uint32_t qbase = 0;
+      for (; ok && w.valid(); w.next(), ++item) {
+        const TcPhase p = w.phase();
+        if (w.ph != cur_ph) {
+          cur_ph = w.ph;
+          ++lp;
+          if (!mbar_wait(bar(BAR_QFULL + (lp & 1)), (lp >> 1) & 1, s_abort, 21, true)) { ok = false; break; }
+          qbase = sbase + SM_Q + (uint32_t)(lp & 1) * Q_BUF_BYTES;
         }
-        for (int t = 0; t < u.ntiles; ++t, ++tile_iter) {
-          const int s = tile_iter % NSTAGE, acc = tile_iter & 1;
-          if (!mbar_wait(bar(BAR_TEMPTY + acc), ((tile_iter >> 1) & 1) ^ 1, s_abort, 22, true)) { ok = false; break; }
-          if (!mbar_wait(bar(BAR_FULL + s), (tile_iter / NSTAGE) & 1, s_abort, 23, true)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t kbase = sbase + SM_K + s * STAGE_BYTES;
-          const uint32_t d0 = tmem + (uint32_t)(acc * 256);
-          if (PASS == 2) {
+        const int s = item % NSTAGE, acc = item & 1;
+        if (!mbar_wait(bar(BAR_TEMPTY + acc), ((item >> 1) & 1) ^ 1, s_abort, 22, true)) { ok = false; break; }
+        if (!mbar_wait(bar(BAR_FULL + s), (item / NSTAGE) & 1, s_abort, 23, true)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t kbase = sbase + SM_K + s * STAGE_BYTES;
+        const uint32_t d0 = tmem + (uint32_t)(acc * 256);
+        if (p.pass == 2) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t ad = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
+            const uint64_t bd = smem_desc(qbase + (ks >> 2) * Q_BLOCK_BYTES + (ks & 3) * 32);
+            tc_mma(d0, ad, bd, idesc2, ks > 0);
+          }
+        } else {
+          for (int hf = 0; hf < nhalf; ++hf) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t ad = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
-              const uint64_t bd = smem_desc(sbase + SM_Q + (ks >> 2) * Q_BLOCK_BYTES + (ks & 3) * 32);
-              tc_mma(d0, ad, bd, idesc, ks > 0);
-            }
-          } else {
-            for (int hf = 0; hf < nhalf; ++hf) {
-#pragma unroll
-              for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t ad = smem_desc(sbase + SM_Q + (ks >> 2) * Q_BLOCK_BYTES + hf * (128 * 128) + (ks & 3) * 32);
-                const uint64_t bd = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
-                tc_mma(d0 + (uint32_t)(hf * 128), ad, bd, idesc, ks > 0);
-              }
+              const uint64_t ad = smem_desc(qbase + (ks >> 2) * Q_BLOCK_BYTES + hf * (128 * 128) + (ks & 3) * 32);
+              const uint64_t bd = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
+              tc_mma(d0 + (uint32_t)(hf * 128), ad, bd, idesc1, ks > 0);
             }
           }
-          tc_commit(bar(BAR_EMPTY + s));       // smem stage free once these MMAs have read it
-          tc_commit(bar(BAR_TFULL + acc));     // accumulator ready for the epilogue
         }
-        const int nxt = ui + gridDim.x;
-        const int next_seg = (nxt < a.n_units) ? a.units[nxt].seg : -1;
-        if (ok && next_seg != cur_seg) tc_commit(bar(BAR_QEMPTY));
+        tc_commit(bar(BAR_EMPTY + s));       // smem stage free once these MMAs have read it
+        tc_commit(bar(BAR_TFULL + acc));     // accumulator ready for the epilogue
+        if (w.last_in_phase()) tc_commit(bar(BAR_QEMPTY + (lp & 1)));   // last tile of the phase here
       }
       if (!ok) {  // make sure nothing is still writing tensor memory before it is freed
         tc_commit(bar(BAR_DRAIN));
         mbar_wait(bar(BAR_DRAIN), 0, s_abort, 24, false);
       }
     }
+  } else if (warp < 4) {
+    // =============================== partial folding ==============================
+    // For every segment, in phase order: wait until all its epilogue sets have
+    // published, then fold the partials of this CTA's rows in a fixed order (the
+    // result does not depend on timing) and count the rows as done.
+    const int hw = warp - 2;
+    const int grid = (int)gridDim.x;
+    const int entries = 2 * grid;                                  // entry e: CTA e/2, set e%2
+    for (int ph = 0; ph < a.n_phases; ++ph) {
+      const TcPhase p = a.phases[ph];
+      if (p.pass != 1) continue;
+      if ((int)blockIdx.x + hw * grid >= NC) continue;             // no row of this segment is ours
+      if (!word_wait(a.published + p.seg, a.epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 2048)) break;
+      const int first = p.g0 % grid;
+      for (int row = blockIdx.x + hw * grid; row < NC; row += 2 * grid) {
+        const float2* src = a.partials + (int64_t)p.seg * entries * NC + row;
+        auto fetch = [&](int e) {
+          int d = (e >> 1) - first;
+          if (d < 0) d += grid;
+          return (e < entries && d < p.ntiles) ? __ldcg(src + (int64_t)e * NC) : make_float2(-INFINITY, 0.f);
+        };
+        float M = -INFINITY, L = 0.f;
+        for (int e0 = 0; e0 < entries; e0 += 320) {
+          float2 v[10];
+#pragma unroll
+          for (int i = 0; i < 10; ++i) v[i] = fetch(e0 + lane + 32 * i);      // all loads in flight
+#pragma unroll
+          for (int i = 0; i < 10; ++i) {
+            if (v[i].y > 0.f) {
+              const float Mn = fmaxf(M, v[i].x);
+              L = L * ex2(M - Mn) + v[i].y * ex2(v[i].x - Mn);
+              M = Mn;
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {                         // butterfly: every lane ends with the same (M, L)
+          const float Mo = __shfl_xor_sync(0xffffffffu, M, o), Lo = __shfl_xor_sync(0xffffffffu, L, o);
+          const bool lower = (lane & o) == 0;                      // fold in lane order so both partners agree bitwise
+          const float Ma = lower ? M : Mo, La = lower ? L : Lo, Mb = lower ? Mo : M, Lb = lower ? Lo : L;
+          const float Mn = fmaxf(Ma, Mb);
+          float Ln = 0.f;
+          if (La > 0.f) Ln += La * ex2(Ma - Mn);
+          if (Lb > 0.f) Ln += Lb * ex2(Mb - Mn);
+          M = Mn; L = Ln;
+        }
+        if (lane == 0) {
+          __stcg(a.offsets + (int64_t)p.seg * NC + row, M + log2f(L));
+          __threadfence();
+          atomicAdd(a.folded + p.seg, 1u);
+        }
+      }
+    }
   } else {
     // =============================== epilogue ===================================
-    const int ew = warp - 2;
-    const int half = ew >> 2;           // which half of the columns (or rows) this warp takes
+    const int set = (warp - 4) >> 2;    // tiles item%2 == set, accumulator `set`
     const int quarter = warp & 3;       // TMEM lanes 32*quarter .. +31 are this warp's
-    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const int st = quarter * 32 + lane;                        // thread of the set, 0..127
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 256);
     const float scale = a.scale_log2;
-    int tile_iter = 0, cur_seg = -1, unit_iter = 0;
-    bool ok = true;
-    for (int ui = blockIdx.x; ok && ui < a.n_units; ui += gridDim.x, ++unit_iter) {
-      const TcUnit u = a.units[ui];
-      const AslReq rq = a.req[u.b];
-      if (PASS == 2 && u.seg != cur_seg) {
-        epi_sync();                                 // everyone is done with the previous offsets
-        const float* off = a.offsets + ((int64_t)u.b * a.Hk + u.h) * a.R + u.chunk * NC;
-        for (int i = threadIdx.x - 64; i < NC; i += 256) s_negoff[i] = -off[i];
-        epi_sync();
-      }
-      cur_seg = u.seg;
-
-      if (PASS == 1) {
-        const int nhalf = (NC > 128) ? 2 : 1;
-        const int ncb = (nhalf == 2) ? 4 : 2;                       // 32-column blocks this thread reads per tile
-        const int col0 = (nhalf == 2) ? half * 128 : half * 64;     // first accumulator column
-        const int key0 = (nhalf == 2) ? 0 : half * 64;              // key offset of that column inside the tile
-        const int row = (nhalf == 2) ? half * 128 + quarter * 32 + lane : quarter * 32 + lane;
-        const bool live = row < NC;
-        const int last = rq.T + (u.chunk * NC + row) % a.W;         // last key this row sees
-        float m = -INFINITY, l = 0.f;
-        for (int t = 0; t < u.ntiles; ++t, ++tile_iter) {
-          const int acc = tile_iter & 1;
-          ok = mbar_wait(bar(BAR_TFULL + acc), (tile_iter >> 1) & 1, s_abort, 31, false);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
-          const int jt = (u.tile0 + t) * KT + key0;
-          for (int cb = 0; cb < ncb; ++cb) {
-            float v[32];
-            tc_ld32(lane_addr + (uint32_t)(acc * 256 + col0 + cb * 32), v);
-            if (!live) continue;
-            const int j0 = jt + cb * 32;
-            if (j0 > last) continue;
-            if (j0 + 31 > last) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) v[i] = (j0 + i <= last) ? v[i] : -INFINITY;
-            }
-            float cmax = v[0];
-#pragma unroll
-            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
-            cmax *= scale;
-            if (cmax > m) { l *= ex2(m - cmax); m = cmax; }
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              s0 += ex2(fmaf(v[i], scale, -m));
-              s1 += ex2(fmaf(v[i + 1], scale, -m));
-            }
-            l += s0 + s1;
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + acc));
-        }
-        if (!ok) break;
-        float2* out = a.partials + (int64_t)ui * NC;
-        if (nhalf == 2) {
-          out[row] = make_float2(m, l);
+    const f32x2 scale2 = pk(scale, scale);
+    float* negoff = s_negoff + set * 256;
+    const int nhalf = (NC > 128) ? 2 : 1;
+    ItemWalk w(a);
+    int item = 0, cur_ph = -1, mine = 0;    // `mine`: tiles this set has taken
+    bool dead = false;                      // a wait expired: keep the barrier sequence, skip the work
+    // pass-1 state of rows st and st + 128: sum of 2^(x - mref) over the keys seen so far.  mref is the
+    // maximum of the first block the row met; later blocks do not track the maximum (their terms may
+    // exceed 1, fp32 has the range), unless a sum overflows, in which case the block is redone with it.
+    float mref0 = -INFINITY, mref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    AslReq rq = a.req[0];
+    for (; w.valid(); w.next(), ++item) {
+      const TcPhase p = w.phase();
+      if (w.ph != cur_ph) {
+        cur_ph = w.ph;
+        rq = a.req[p.b];
+        if (p.pass == 1) {
+          mref0 = mref1 = -INFINITY;
+          l0 = l1 = 0.f;
         } else {
-          float2* sc = s_scratch + (unit_iter & 1) * 256;
-          sc[half * 128 + quarter * 32 + lane] = make_float2(m, l);
-          epi_sync();
-          if (half == 0 && live) {
-            const float2 o = sc[128 + row];
-            const float M = fmaxf(m, o.x);
-            float L = 0.f;
-            if (l > 0.f) L += l * ex2(m - M);
-            if (o.y > 0.f) L += o.y * ex2(o.x - M);
-            out[row] = make_float2(M, L);
-          }
+          // the segment's offsets: wait until every row has been folded, then stage -offset for this set
+          if (!dead) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
+          bar_sync(2 + set, 128);                                 // the set is done with the previous offsets
+          const float* off = a.offsets + (int64_t)p.seg * NC;
+          for (int i = st; i < NC; i += 128) negoff[i] = dead ? 0.f : -__ldcg(off + i);
+          bar_sync(2 + set, 128);
         }
-      } else {
-        // ---- pass 2 ----
-        const int hc = NC >> 1;                                   // columns per half
-        const int cw = a.W < hc ? a.W : hc;                       // columns of one query head inside a half
-        const int nslot = PER_Q ? hc / cw : 1;
-        const bool combine = !PER_Q || a.W > hc;                  // both halves feed the same output row
-        const int key_lane = quarter * 32 + lane;
-        for (int t = 0; t < u.ntiles; ++t, ++tile_iter) {
-          const int acc = tile_iter & 1;
-          ok = mbar_wait(bar(BAR_TFULL + acc), (tile_iter >> 1) & 1, s_abort, 32, false);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
+      }
+      if ((item & 1) == set) {
+        if (!dead) {
+          const bool ok = mbar_wait(bar(BAR_TFULL + set), mine & 1, s_abort, 31, true);
+          dead = !__all_sync(0xffffffffu, ok);
+        }
+        ++mine;
+        if (!dead) {
           tc_fence_after();
-          float sums[4] = {0.f, 0.f, 0.f, 0.f};
-          const int ncb = hc / 32;
-          for (int cb = 0; cb < ncb; ++cb) {
-            float v[32];
-            const int c0 = half * hc + cb * 32;
-            tc_ld32(lane_addr + (uint32_t)(acc * 256 + c0), v);
-            const float4* no = reinterpret_cast<const float4*>(s_negoff + c0);
-            float s0 = 0.f, s1 = 0.f;
+          const int tile = w.g - p.g0;
+          // The accumulator is read 32 columns at a time into two register buffers: the load of
+          // block i+1 is in flight while block i is processed.  The loop over blocks stays rolled
+          // (two blocks per trip) so that the code fits the instruction cache.
+          uint32_t b0[32], b1[32];
+          auto release = [&]() {                                   // accumulator fully read: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + set));
+          };
+          if (p.pass == 1) {
+            // ---- pass 1: sum of 2^(x - mref) of this thread's rows over the tile's 128 keys ----
+            const int nblk = 4 * nhalf;
+            auto block1 = [&](const uint32_t(&cur)[32], int blk) {
+              const int hf = blk >> 2;
+              const int j0 = tile * KT + (blk & 3) * 32;
+              float mr = hf ? mref1 : mref0;
+              float ls = hf ? l1 : l0;
+              bool careful = (mr == -INFINITY) || (j0 + 31 > rq.T);    // first block of the row, or window keys inside
+              if (!careful) {
+                const f32x2 nm2 = pk(-mr, -mr);
+                const float bs = exp_sum32(cur, scale2, [&](int) { return nm2; });
+                if (bs < INFINITY) ls += bs;
+                else careful = true;                                  // a term overflowed: redo with the maximum
+              }
+              if (careful) {
+                const int row = hf * 128 + st;
+                const int lastkey = rq.T + (p.chunk * NC + row) % a.W;     // last key this row sees
+                if (j0 <= lastkey) {
+                  float c = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float4 o = no[i];
-              s0 += ex2(fmaf(v[4 * i + 0], scale, o.x));
-              s1 += ex2(fmaf(v[4 * i + 1], scale, o.y));
-              s0 += ex2(fmaf(v[4 * i + 2], scale, o.z));
-              s1 += ex2(fmaf(v[4 * i + 3], scale, o.w));
-            }
-            const int slot = PER_Q ? (cb * 32) / cw : 0;
-            sums[slot & 3] += s0 + s1;
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + acc));
-          const int j = (u.tile0 + t) * KT + key_lane;
-          if (combine) {
-            float* hs = reinterpret_cast<float*>(s_scratch) + acc * 128;
-            if (half == 1) hs[key_lane] = sums[0];
-            epi_sync();
-            if (half == 0 && j < rq.T) {
-              const int row_u = PER_Q ? (u.h * a.G + (u.chunk * NC) / a.W) : (u.h * a.u_rows_per_kv + u.chunk);
-              a.u[(int64_t)row_u * a.sum_T + rq.t_off + j] = sums[0] + hs[key_lane];
-            }
-          } else if (j < rq.T) {
+                  for (int i = 0; i < 32; ++i) c = fmaxf(c, (j0 + i <= lastkey) ? __uint_as_float(cur[i]) : -INFINITY);
+                  const float mn = fmaxf(mr, c * scale);
+                  float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              if (q < nslot) {
-                const int head = u.h * a.G + (u.chunk * NC + half * hc + q * cw) / a.W;
-                a.u[(int64_t)head * a.sum_T + rq.t_off + j] = sums[q];
+                  for (int i = 0; i < 32; i += 2) {
+                    s0 += (j0 + i <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i]), scale, -mn)) : 0.f;
+                    s1 += (j0 + i + 1 <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -mn)) : 0.f;
+                  }
+                  ls = fmaf(ls, ex2(mr - mn), s0 + s1);
+                  mr = mn;
+                }
+              }
+              if (ls > 0x1p60f) { ls *= 0x1p-60f; mr += 60.f; }       // exact: keeps the running sum far from overflow
+              if (hf) { mref1 = mr; l1 = ls; } else { mref0 = mr; l0 = ls; }
+            };
+            tc_ld32_issue(lane_addr, b0);
+            tc_ld_wait(b0);
+#pragma unroll 1
+            for (int blk = 0; blk < nblk; blk += 2) {
+              tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
+              block1(b0, blk);
+              tc_ld_wait(b1);
+              const bool more = blk + 2 < nblk;
+              if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
+              else release();
+              block1(b1, blk + 1);
+              if (more) tc_ld_wait(b0);
+            }
+          } else {
+            // ---- pass 2: this thread's key, exp2(x - offset[row]) summed over the chunk's rows ----
+            const int nblk = NC >> 5;
+            float sums[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) sums[q] = 0.f;
+            auto block2 = [&](const uint32_t(&cur)[32], int blk) {
+              const float4* no = reinterpret_cast<const float4*>(negoff + blk * 32);
+              float4 o[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) o[i] = no[i];
+              const float bs = exp_sum32(cur, scale2, [&](int pi) {
+                const float4 v = o[pi >> 1];
+                return (pi & 1) ? pk(v.z, v.w) : pk(v.x, v.y);
+              });
+              if (PER_Q) {                                         // W is a multiple of 32: a block never straddles heads
+                const int slot = (blk * 32) / a.W;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) sums[q] += (q == slot) ? bs : 0.f;
+              } else {
+                sums[0] += bs;
+              }
+            };
+            tc_ld32_issue(lane_addr, b0);
+            tc_ld_wait(b0);
+#pragma unroll 1
+            for (int blk = 0; blk < nblk; blk += 2) {
+              tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
+              block2(b0, blk);
+              tc_ld_wait(b1);
+              const bool more = blk + 2 < nblk;
+              if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
+              else release();
+              block2(b1, blk + 1);
+              if (more) tc_ld_wait(b0);
+            }
+            const int j = tile * KT + st;
+            if (j < rq.T) {
+              if (PER_Q) {
+                const int nslot = NC / a.W;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  if (q < nslot) {
+                    const int head = p.h * a.G + (p.chunk * NC) / a.W + q;
+                    a.u[(int64_t)head * a.sum_T + rq.t_off + j] = sums[q];
+                  }
+                }
+              } else {
+                a.u[(int64_t)(p.h * a.u_rows_per_kv + p.chunk) * a.sum_T + rq.t_off + j] = sums[0];
               }
             }
           }
         }
-        if (!ok) break;
+      }
+      if (w.last_in_phase() && p.pass == 1) {
+        // ---- end of a pass-1 phase in this CTA: each set publishes its own (reference, sum) per row ----
+        float2* out = a.partials + (((int64_t)p.seg * gridDim.x + blockIdx.x) * 2 + set) * NC;
+        if (st < NC) __stcg(out + st, make_float2(mref0, dead ? 0.f : l0));
+        if (128 + st < NC) __stcg(out + 128 + st, make_float2(mref1, dead ? 0.f : l1));
+        __threadfence();
+        bar_sync(2 + set, 128);
+        if (st == 0) atomicAdd(a.published + p.seg, 1u);
       }
     }
   }
@@ -439,23 +702,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
-  if (threadIdx.x == 0 && *s_abort) atomicCAS(a.err, 0, *s_abort + 100 * PASS);
-}
-
-// offset[row] = max + log2(sum) over the units of the row's (request, head, chunk), in unit order
-__global__ void __launch_bounds__(256) score_tc_combine(const float2* __restrict__ partials, const TcSeg* __restrict__ segs,
-                                                        int NC, int Hk, int R, float* __restrict__ offsets) {
-  const TcSeg sg = segs[blockIdx.x];
-  for (int c = threadIdx.x; c < NC; c += blockDim.x) {
-    float M = -INFINITY;
-    for (int i = 0; i < sg.nunits; ++i) M = fmaxf(M, partials[(int64_t)(sg.unit0 + i) * NC + c].x);
-    float L = 0.f;
-    for (int i = 0; i < sg.nunits; ++i) {
-      const float2 p = partials[(int64_t)(sg.unit0 + i) * NC + c];
-      if (p.y > 0.f) L += p.y * exp2f(p.x - M);
-    }
-    offsets[((int64_t)sg.b * Hk + sg.h) * R + sg.chunk * NC + c] = M + log2f(L);
-  }
+  if (threadIdx.x == 0 && *s_abort) atomicCAS(a.err, 0, *s_abort);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -492,76 +739,78 @@ bool asl_tc_plan(asl_ctx* c) {
   AslTcPlan& tp = c->tc;
   tp = AslTcPlan();
   const int W = p.window, G = p.n_q_heads / p.n_kv_heads, R = G * W;
-  if (p.head_dim != 128 || W % 32) return false;
+  if (p.head_dim != 128 || W % 32 || W > MAX_NC) return false;
   int NC = 0;
-  if (W <= 256) {
-    for (int m = 256 / W; m >= 1; --m)
-      if (R % (m * W) == 0) { NC = m * W; break; }
-  } else {
-    for (int cnd = 256; cnd >= 64; cnd -= 64)
-      if (W % cnd == 0) { NC = cnd; break; }
-  }
+  for (int m = MAX_NC / W; m >= 1; --m)
+    if (R % (m * W) == 0) { NC = m * W; break; }
   if (NC < 64 || NC % 64 || R % NC) return false;
-  if (p.pool_mode == ASL_POOL_MAX) {            // per-query-head sums: at most 4 heads per column half
-    const int hc = NC / 2, cw = W < hc ? W : hc;
-    if (hc / cw > 4) return false;
-  }
   tp.NC = NC;
   tp.nchunk = R / NC;
-  int64_t tiles1 = 0, tiles2 = 0;
-  for (const AslReq& r : c->req) {
-    tiles1 += (int64_t)p.n_kv_heads * tp.nchunk * ((r.n + KT - 1) / KT);
-    tiles2 += (int64_t)p.n_kv_heads * tp.nchunk * ((r.T + KT - 1) / KT);
-  }
-  auto build = [&](bool past_only, int64_t total_tiles, std::vector<TcUnit>& units, std::vector<TcSeg>& segs) {
-    int64_t tps = (total_tiles + 4 * c->sm_count - 1) / (4 * (int64_t)c->sm_count);
-    if (tps < 2) tps = 2;
-    if (tps > 32) tps = 32;
-    for (int b = 0; b < p.batch; ++b) {
-      const int len = past_only ? c->req[b].T : c->req[b].n;
-      const int tiles = (len + KT - 1) / KT;
-      for (int h = 0; h < p.n_kv_heads; ++h)
-        for (int ch = 0; ch < tp.nchunk; ++ch) {
-          TcSeg sg{};
-          sg.unit0 = (int32_t)units.size(); sg.b = b; sg.h = h; sg.chunk = ch;
-          for (int t0 = 0, split = 0; t0 < tiles; t0 += (int)tps, ++split) {
-            TcUnit u{};
-            u.b = b; u.h = h; u.chunk = ch; u.tile0 = t0;
-            u.ntiles = (int32_t)((tiles - t0) < tps ? (tiles - t0) : tps);
-            u.seg = (int32_t)segs.size(); u.split = split;
-            units.push_back(u);
-          }
-          sg.nunits = (int32_t)units.size() - sg.unit0;
-          segs.push_back(sg);
-        }
-    }
+  tp.grid = c->sm_count;
+
+  // segments in (request, head, chunk) order; phases in groups: pass 1 of `group` segments, then their pass 2
+  struct Seg { int b, h, chunk, tiles1, tiles2; };
+  std::vector<Seg> segs;
+  for (int b = 0; b < p.batch; ++b)
+    for (int h = 0; h < p.n_kv_heads; ++h)
+      for (int ch = 0; ch < tp.nchunk; ++ch)
+        segs.push_back({b, h, ch, (c->req[b].n + KT - 1) / KT, (c->req[b].T + KT - 1) / KT});
+  tp.nseg = (int)segs.size();
+  const int group = c->score_group > 0 ? c->score_group : 2;
+  tp.group = group;
+  int64_t g = 0;
+  auto push = [&](int s, int pass) {
+    TcPhase ph{};
+    ph.g0 = (int32_t)g;
+    ph.ntiles = pass == 1 ? segs[s].tiles1 : segs[s].tiles2;
+    ph.pass = pass; ph.seg = s; ph.b = segs[s].b; ph.h = segs[s].h; ph.chunk = segs[s].chunk;
+    ph.ncontrib = segs[s].tiles1 < tp.grid ? segs[s].tiles1 : tp.grid;    // CTAs with a tile in pass 1
+    g += ph.ntiles;
+    tp.phases.push_back(ph);
   };
-  std::vector<TcSeg> segs2;
-  build(false, tiles1, tp.units1, tp.segs1);
-  build(true, tiles2, tp.units2, segs2);
-  cudaError_t e = cudaMalloc(&tp.d_units1, tp.units1.size() * sizeof(TcUnit));
-  if (e == cudaSuccess) e = cudaMalloc(&tp.d_units2, tp.units2.size() * sizeof(TcUnit));
-  if (e == cudaSuccess) e = cudaMalloc(&tp.d_segs1, tp.segs1.size() * sizeof(TcSeg));
-  if (e == cudaSuccess) e = cudaMemcpy(tp.d_units1, tp.units1.data(), tp.units1.size() * sizeof(TcUnit), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemcpy(tp.d_units2, tp.units2.data(), tp.units2.size() * sizeof(TcUnit), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemcpy(tp.d_segs1, tp.segs1.data(), tp.segs1.size() * sizeof(TcSeg), cudaMemcpyHostToDevice);
+  for (int s0 = 0; s0 < tp.nseg; s0 += group) {
+    const int s1 = s0 + group < tp.nseg ? s0 + group : tp.nseg;
+    for (int s = s0; s < s1; ++s) push(s, 1);
+    for (int s = s0; s < s1; ++s) push(s, 2);
+  }
+  if (g >= ((int64_t)1 << 31) - tp.grid) return false;
+  tp.total_items = (int32_t)g;
+
+  const size_t sync_bytes = 2 * (size_t)tp.nseg * sizeof(uint32_t);
+  cudaError_t e = cudaMalloc(&tp.d_phases, tp.phases.size() * sizeof(TcPhase));
+  if (e == cudaSuccess) e = cudaMalloc(&tp.d_sync, sync_bytes);
+  if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases, tp.phases.data(), tp.phases.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(tp.d_sync, 0, sync_bytes);
   if (e != cudaSuccess) { asl_tc_free(c); return false; }
-  cudaFuncSetAttribute(score_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  cudaFuncSetAttribute(score_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  cudaFuncSetAttribute(score_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  tp.epoch = 0;
+  cudaFuncSetAttribute(score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaFuncSetAttribute(score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (cudaGetLastError() != cudaSuccess) { asl_tc_free(c); return false; }
   tp.enabled = encode_fn() != nullptr;
   return tp.enabled;
 }
 
+size_t asl_tc_partial_bytes(const asl_ctx* c) {
+  const AslTcPlan& tp = c->tc;
+  return (size_t)tp.nseg * tp.grid * 2 * tp.NC * sizeof(float2);
+}
+
 void asl_tc_free(asl_ctx* c) {
   AslTcPlan& tp = c->tc;
-  if (tp.d_units1) cudaFree(tp.d_units1);
-  if (tp.d_units2) cudaFree(tp.d_units2);
-  if (tp.d_segs1) cudaFree(tp.d_segs1);
-  tp.d_units1 = tp.d_units2 = nullptr;
-  tp.d_segs1 = nullptr;
+  if (tp.d_phases) cudaFree(tp.d_phases);
+  if (tp.d_sync) cudaFree(tp.d_sync);
+  tp.d_phases = nullptr;
+  tp.d_sync = nullptr;
   tp.enabled = false;
+}
+
+// after a reported device error the publish counters may be inconsistent: start over
+asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st) {
+  AslTcPlan& tp = c->tc;
+  if (!tp.d_sync) return ASL_OK;
+  ASL_CUDA(cudaMemsetAsync(tp.d_sync, 0, 2 * (size_t)tp.nseg * sizeof(uint32_t), st));
+  tp.epoch = 0;
+  return ASL_OK;
 }
 
 asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg, char* ws,
@@ -583,30 +832,32 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* 
     const cuuint32_t box[3] = {64, 1, (cuuint32_t)KT};
     if (!make_map(&tm_k, k, 3, dims, strides, box)) return ASL_ERR_CUDA;
   }
+  if (tp.epoch >= 0xFFFFFFFFu / (uint32_t)(2 * tp.grid > MAX_NC ? 2 * tp.grid : MAX_NC) - 1u) {   // the counters would wrap
+    const asl_status rs = asl_tc_reset_sync(c, st);
+    if (rs != ASL_OK) return rs;
+  }
   TcArgs a{};
+  a.phases = tp.d_phases;
   a.req = c->d_req;
   a.partials = reinterpret_cast<float2*>(ws + c->ws.score_partials);
-  float* offsets = reinterpret_cast<float*>(ws + c->ws.score_offsets);
+  a.offsets = reinterpret_cast<float*>(ws + c->ws.score_offsets);
   float* u = reinterpret_cast<float*>(ws + c->ws.score_u);
-  a.offsets = offsets;
   a.u = u;
+  a.published = tp.d_sync;
+  a.folded = tp.d_sync + tp.nseg;
   a.err = c->d_err;
   a.sum_T = c->sum_T;
-  a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads; a.R = c->rows_per_kv;
+  a.epoch = ++tp.epoch;
+  a.n_phases = (int32_t)tp.phases.size();
+  a.total_items = tp.total_items;
+  a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads;
   a.u_rows_per_kv = c->u_rows_per_kv;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.head_dim));
-  const int grid = c->sm_count;
-
-  a.units = tp.d_units1;
-  a.n_units = (int32_t)tp.units1.size();
-  score_tc_kernel<1, false><<<grid < a.n_units ? grid : a.n_units, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
-  score_tc_combine<<<(unsigned)tp.segs1.size(), 256, 0, st>>>(a.partials, tp.d_segs1, NC, a.Hk, a.R, offsets);
-  a.units = tp.d_units2;
-  a.n_units = (int32_t)tp.units2.size();
-  const int g2 = grid < a.n_units ? grid : a.n_units;
-  if (p.pool_mode == ASL_POOL_MAX) score_tc_kernel<2, true><<<g2, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
-  else                             score_tc_kernel<2, false><<<g2, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
-  c->launches += 3;
+  // every CTA must be resident at once (pass 2 waits for counters other CTAs advance): one CTA per SM at most
+  const int grid = tp.grid;
+  if (p.pool_mode == ASL_POOL_MAX) score_tc_kernel<true><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+  else                             score_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+  c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return asl_launch_pool(c, u, scores_kv, scores_agg, st);
 }

@@ -1,22 +1,24 @@
-// Plan of the tensor-core scorer: work units and segments built at plan time.
+// Plan of the tensor-core scorer: the phase list built at plan time.
 #pragma once
 #include <stdint.h>
 #include <vector>
 
 constexpr int ASL_TC_KEY_TILE = 128;
 
-// a run of consecutive key tiles of one (request, kv head, row chunk)
-struct TcUnit { int32_t b, h, chunk, tile0, ntiles, seg, split, pad; };
-// all units of one (request, kv head, row chunk)
-struct TcSeg { int32_t unit0, nunits, b, h, chunk, pad0, pad1, pad2; };
+// one pass over the 128-key tiles of one segment = (request, kv head, row chunk);
+// its tiles are the global work items g0 .. g0 + ntiles - 1
+struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib; };
 
 struct AslTcPlan {
   bool enabled = false;
-  int NC = 0;         // query rows per chunk (MMA N in pass 2)
-  int nchunk = 0;     // chunks per kv head
-  std::vector<TcUnit> units1, units2;   // pass 1 (all keys), pass 2 (past keys)
-  std::vector<TcSeg> segs1;
-  TcUnit* d_units1 = nullptr;
-  TcUnit* d_units2 = nullptr;
-  TcSeg* d_segs1 = nullptr;
+  int NC = 0;           // query rows per chunk (MMA N in pass 2)
+  int nchunk = 0;       // chunks per kv head
+  int nseg = 0;         // segments
+  int grid = 0;         // CTAs of the persistent kernel (one per SM)
+  int group = 0;        // segments whose pass 1 runs before their pass 2
+  int32_t total_items = 0;
+  uint32_t epoch = 0;   // launches so far; the device counters accumulate over launches
+  std::vector<TcPhase> phases;
+  TcPhase* d_phases = nullptr;
+  uint32_t* d_sync = nullptr;   // [nseg] publish counters, [nseg] folded-row counters
 };
