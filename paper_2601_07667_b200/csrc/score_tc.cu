@@ -295,19 +295,26 @@ struct TcArgs {
   float scale_log2;
 };
 
-// walks the CTA's items (global item g = blockIdx.x + i*gridDim.x) through the phase list;
-// the current phase record stays in registers and is re-read only when g leaves it
+// walks the CTA's items (global item g = blockIdx.x + i*gridDim.x) through the phase list.  The
+// current phase record and the one after it stay in registers: the next record is requested when a
+// phase is entered, so its load latency is hidden behind the phase's tiles.
 struct ItemWalk {
   const TcPhase* phases;
-  int total;
+  int total, n_phases;
   int g, ph;
-  TcPhase cur;
-  __device__ __forceinline__ ItemWalk(const TcArgs& a) : phases(a.phases), total(a.total_items), g((int)blockIdx.x), ph(0) {
+  TcPhase cur, nxt;
+  __device__ __forceinline__ ItemWalk(const TcArgs& a) : phases(a.phases), total(a.total_items), n_phases(a.n_phases),
+                                                       g((int)blockIdx.x), ph(0) {
     cur = phases[0];
+    nxt = phases[n_phases > 1 ? 1 : 0];
   }
   __device__ __forceinline__ bool valid() const { return g < total; }
   __device__ __forceinline__ const TcPhase& phase() {       // phases are sorted by g0 and cover [0, total)
-    while (g >= cur.g0 + cur.ntiles) cur = phases[++ph];
+    while (g >= cur.g0 + cur.ntiles) {
+      cur = nxt;
+      ++ph;
+      nxt = phases[ph + 1 < n_phases ? ph + 1 : ph];
+    }
     return cur;
   }
   __device__ __forceinline__ bool last_in_phase() const { return g + (int)gridDim.x >= cur.g0 + cur.ntiles; }
@@ -391,7 +398,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (w.ph != cur_ph) {
           cur_ph = w.ph;
           ++lp;
-          tok_off = a.req[p.b].tok_off;
+          tok_off = p.tok_off;
           if (q_issued < lp && !issue_q(lp, p, true)) { ok = false; break; }
           // where does this CTA go after this phase?
           const int end = p.g0 + p.ntiles;
@@ -541,18 +548,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     int item = 0, cur_ph = -1, mine = 0;    // `mine`: tiles this set has taken
     bool dead = false;                      // a wait expired: keep the barrier sequence, skip the work
     // pass-1 state of rows st and st + 128: sum of 2^(x - mref) over the keys seen so far.  mref is the
-    // maximum of the first block the row met; later blocks do not track the maximum (their terms may
-    // exceed 1, fp32 has the range), unless a sum overflows, in which case the block is redone with it.
+    // maximum of the first 32 keys the row met; later blocks do not track the maximum (their terms may
+    // exceed 1, fp32 has the range), unless a sum overflows, in which case the tile is redone with it.
     float mref0 = -INFINITY, mref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-    AslReq rq = a.req[0];
+    bool first_tile = true;                 // this set has not yet taken a tile of the current pass-1 phase
     for (; w.valid(); w.next(), ++item) {
       const TcPhase p = w.phase();
       if (w.ph != cur_ph) {
         cur_ph = w.ph;
-        rq = a.req[p.b];
         if (p.pass == 1) {
           mref0 = mref1 = -INFINITY;
           l0 = l1 = 0.f;
+          first_tile = true;
         } else {
           // the segment's offsets: wait until every row has been folded, then stage -offset for this set
           if (!dead) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
@@ -582,23 +589,56 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           };
           if (p.pass == 1) {
             // ---- pass 1: sum of 2^(x - mref) of this thread's rows over the tile's 128 keys ----
+            // Fast walk: every key of the tile is visible to every row; it does not track the maximum.
+            // Careful walk (tiles that reach into the window, or after a sum overflowed in the fast
+            // walk): per-row masks, block maxima, MUFU only.  The two walks are separate loops so that the rare one costs the
+            // common one nothing.
             const int nblk = 4 * nhalf;
-            auto block1 = [&](const uint32_t(&cur)[32], int blk) {
-              const int hf = blk >> 2;
-              const int j0 = tile * KT + (blk & 3) * 32;
-              float mr = hf ? mref1 : mref0;
-              float ls = hf ? l1 : l0;
-              bool careful = (mr == -INFINITY) || (j0 + 31 > rq.T);    // first block of the row, or window keys inside
-              if (!careful) {
+            const float keep_m0 = mref0, keep_m1 = mref1, keep_l0 = l0, keep_l1 = l1;
+            bool careful = tile * KT + KT - 1 > p.T;
+            if (!careful) {
+              auto block1 = [&](const uint32_t(&cur)[32], int blk) {
+                const bool hf = blk >= 4;
+                if (first_tile && (blk & 3) == 0) {               // first block of these rows: its maximum is the reference
+                  float c0 = fmaxf(__uint_as_float(cur[0]), __uint_as_float(cur[1]));
+                  float c1 = fmaxf(__uint_as_float(cur[2]), __uint_as_float(cur[3]));
+#pragma unroll
+                  for (int i = 4; i < 32; i += 4) {
+                    c0 = fmaxf(c0, fmaxf(__uint_as_float(cur[i]), __uint_as_float(cur[i + 1])));
+                    c1 = fmaxf(c1, fmaxf(__uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3])));
+                  }
+                  if (hf) mref1 = fmaxf(c0, c1) * scale; else mref0 = fmaxf(c0, c1) * scale;
+                }
+                const float mr = hf ? mref1 : mref0;
                 const f32x2 nm2 = pk(-mr, -mr);
                 const float bs = exp_sum32(cur, scale2, [&](int) { return nm2; });
-                if (bs < INFINITY) ls += bs;
-                else careful = true;                                  // a term overflowed: redo with the maximum
+                if (hf) l1 += bs; else l0 += bs;
+              };
+              tc_ld32_issue(lane_addr, b0);
+              tc_ld_wait(b0);
+#pragma unroll 1
+              for (int blk = 0; blk < nblk; blk += 2) {
+                tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
+                block1(b0, blk);
+                tc_ld_wait(b1);
+                const bool more = blk + 2 < nblk;
+                if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
+                block1(b1, blk + 1);
+                if (more) tc_ld_wait(b0);
               }
-              if (careful) {
-                const int row = hf * 128 + st;
-                const int lastkey = rq.T + (p.chunk * NC + row) % a.W;     // last key this row sees
+              // a term beyond fp32 range (a logit 127 above the reference): redo the tile carefully
+              careful = __any_sync(0xffffffffu, !(l0 < INFINITY) || !(l1 < INFINITY));
+              if (careful) { mref0 = keep_m0; mref1 = keep_m1; l0 = keep_l0; l1 = keep_l1; }
+            }
+            if (careful) {
+              auto block1c = [&](const uint32_t(&cur)[32], int blk) {
+                const bool hf = blk >= 4;
+                const int j0 = tile * KT + (blk & 3) * 32;
+                const int row = (hf ? 128 : 0) + st;
+                const int lastkey = p.T + (p.chunk * NC + row) % a.W;       // last key this row sees
                 if (j0 <= lastkey) {
+                  float mr = hf ? mref1 : mref0;
+                  float ls = hf ? l1 : l0;
                   float c = -INFINITY;
 #pragma unroll
                   for (int i = 0; i < 32; ++i) c = fmaxf(c, (j0 + i <= lastkey) ? __uint_as_float(cur[i]) : -INFINITY);
@@ -610,25 +650,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     s1 += (j0 + i + 1 <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -mn)) : 0.f;
                   }
                   ls = fmaf(ls, ex2(mr - mn), s0 + s1);
-                  mr = mn;
+                  if (hf) { mref1 = mn; l1 = ls; } else { mref0 = mn; l0 = ls; }
                 }
-              }
-              if (ls > 0x1p60f) { ls *= 0x1p-60f; mr += 60.f; }       // exact: keeps the running sum far from overflow
-              if (hf) { mref1 = mr; l1 = ls; } else { mref0 = mr; l0 = ls; }
-            };
-            tc_ld32_issue(lane_addr, b0);
-            tc_ld_wait(b0);
+              };
 #pragma unroll 1
-            for (int blk = 0; blk < nblk; blk += 2) {
-              tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
-              block1(b0, blk);
-              tc_ld_wait(b1);
-              const bool more = blk + 2 < nblk;
-              if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
-              else release();
-              block1(b1, blk + 1);
-              if (more) tc_ld_wait(b0);
+              for (int blk = 0; blk < nblk; ++blk) {
+                tc_ld32_issue(lane_addr + (uint32_t)(blk * 32), b0);
+                tc_ld_wait(b0);
+                block1c(b0, blk);
+              }
             }
+            release();
+            // exact rescaling keeps the running sums far from overflow
+            if (l0 > 0x1p60f) { l0 *= 0x1p-60f; mref0 += 60.f; }
+            if (l1 > 0x1p60f) { l1 *= 0x1p-60f; mref1 += 60.f; }
+            first_tile = false;
           } else {
             // ---- pass 2: this thread's key, exp2(x - offset[row]) summed over the chunk's rows ----
             const int nblk = NC >> 5;
@@ -666,18 +702,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               if (more) tc_ld_wait(b0);
             }
             const int j = tile * KT + st;
-            if (j < rq.T) {
+            if (j < p.T) {
               if (PER_Q) {
                 const int nslot = NC / a.W;
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                   if (q < nslot) {
                     const int head = p.h * a.G + (p.chunk * NC) / a.W + q;
-                    a.u[(int64_t)head * a.sum_T + rq.t_off + j] = sums[q];
+                    a.u[(int64_t)head * a.sum_T + p.t_off + j] = sums[q];
                   }
                 }
               } else {
-                a.u[(int64_t)(p.h * a.u_rows_per_kv + p.chunk) * a.sum_T + rq.t_off + j] = sums[0];
+                a.u[(int64_t)(p.h * a.u_rows_per_kv + p.chunk) * a.sum_T + p.t_off + j] = sums[0];
               }
             }
           }
@@ -688,9 +724,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         float2* out = a.partials + (((int64_t)p.seg * gridDim.x + blockIdx.x) * 2 + set) * NC;
         if (st < NC) __stcg(out + st, make_float2(mref0, dead ? 0.f : l0));
         if (128 + st < NC) __stcg(out + 128 + st, make_float2(mref1, dead ? 0.f : l1));
-        __threadfence();
         bar_sync(2 + set, 128);
-        if (st == 0) atomicAdd(a.published + p.seg, 1u);
+        if (st == 0) {                 // the barrier orders the set's stores before this thread's fence: the release is cumulative
+          __threadfence();
+          atomicAdd(a.published + p.seg, 1u);
+        }
       }
     }
   }
@@ -765,6 +803,7 @@ bool asl_tc_plan(asl_ctx* c) {
     ph.ntiles = pass == 1 ? segs[s].tiles1 : segs[s].tiles2;
     ph.pass = pass; ph.seg = s; ph.b = segs[s].b; ph.h = segs[s].h; ph.chunk = segs[s].chunk;
     ph.ncontrib = segs[s].tiles1 < tp.grid ? segs[s].tiles1 : tp.grid;    // CTAs with a tile in pass 1
+    ph.T = c->req[ph.b].T; ph.t_off = c->req[ph.b].t_off; ph.tok_off = c->req[ph.b].tok_off;
     g += ph.ntiles;
     tp.phases.push_back(ph);
   };

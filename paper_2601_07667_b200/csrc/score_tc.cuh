@@ -7,7 +7,9 @@ constexpr int ASL_TC_KEY_TILE = 128;
 
 // one pass over the 128-key tiles of one segment = (request, kv head, row chunk);
 // its tiles are the global work items g0 .. g0 + ntiles - 1
-struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib; };
+// (T, t_off, tok_off: the request's past length, score offset and first token, copied here so that
+// one record is all a role needs when it enters the phase)
+struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, pad; };
 
 struct AslTcPlan {
   bool enabled = false;
