@@ -128,10 +128,13 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
 
   cudaGetDevice(&prev);
   cudaSetDevice(c->device);
-  const bool tc = asl_tc_plan(c);
+  const bool tc = asl_tc_plan(c) && !c->force_simt;
   cudaSetDevice(prev);
   const int G = p->n_q_heads / p->n_kv_heads;
-  c->u_rows_per_kv = p->pool_mode == ASL_POOL_MAX ? G : (tc ? c->tc.nchunk : 1);
+  // the tensor-core scorer writes two partial column sums per chunk (one per half of the chunk's rows);
+  // under max pooling they belong to different query heads unless a chunk is a single head
+  c->u_parts = (tc && p->pool_mode == ASL_POOL_MAX && p->window > c->tc.NC / 2) ? 2 : 1;
+  c->u_rows_per_kv = p->pool_mode == ASL_POOL_MAX ? G * c->u_parts : (tc ? 2 * c->tc.nchunk : 1);
 
   AslWorkspace& w = c->ws;
   size_t off = 0;

@@ -51,7 +51,9 @@ struct asl_ctx {
   // scorer plan
   int32_t rows_per_kv = 0;            // G*W
   int32_t n_key_tiles = 0;            // sum over requests of ceil(n_b / tile)
-  int32_t u_rows_per_kv = 1;          // rows of un-pooled column sums per kv head (chunks, or G for max pooling)
+  int32_t u_rows_per_kv = 1;          // rows of un-pooled column sums per kv head (average pooling: all are added;
+                                      // max pooling: G * u_parts, u_parts consecutive rows per query head)
+  int32_t u_parts = 1;                // partial rows per query head under max pooling
   AslTcPlan tc;                       // tensor-core scorer plan (enabled when the shape fits)
   AslWorkspace ws{};
   int64_t launches = 0;

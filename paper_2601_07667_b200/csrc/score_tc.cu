@@ -26,8 +26,8 @@
 // Inside a CTA: warp 0 streams K tiles through a 3-stage TMA ring (128B-swizzled)
 // and keeps the Q chunks of two phases resident (the next one is prefetched);
 // warp 1 issues tcgen05.mma into two 256-column TMEM accumulators; warps 2-3 fold
-// pass-1 partials; two sets of four epilogue warps take alternate tiles, one
-// accumulator each, reading it with software-pipelined tcgen05.ld.  The
+// pass-1 partials; two sets of eight epilogue warps take alternate tiles, one
+// accumulator each (two warps per TMEM lane quarter, half of the columns each).  The
 // exponentials are split between the MUFU unit and a degree-3 polynomial on the
 // FMA pipe (packed f32x2 arithmetic).
 //
@@ -48,7 +48,7 @@ constexpr int STAGE_BYTES = 2 * HALF_BYTES;
 constexpr int MAX_NC = 256;
 constexpr int Q_BLOCK_BYTES = MAX_NC * 128;  // one 64-channel block of a Q chunk
 constexpr int Q_BUF_BYTES = 2 * Q_BLOCK_BYTES;
-constexpr int THREADS = 384;                 // warp 0: TMA, 1: MMA, 2-3: partial folding, 4-7 / 8-11: epilogue sets
+constexpr int THREADS = 640;                 // warp 0: TMA, 1: MMA, 2-3: partial folding, 4-11 / 12-19: epilogue sets
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // every wait gives up after 2 s
 
 // shared-memory map (offsets from the 1024-aligned base of dynamic shared memory)
@@ -291,7 +291,7 @@ struct TcArgs {
   int32_t* err;
   int64_t sum_T;
   uint32_t epoch;          // launch number, from 1
-  int32_t n_phases, total_items, NC, W, G, Hk, u_rows_per_kv;
+  int32_t n_phases, total_items, NC, W, G, Hk, u_rows_per_kv, u_parts;
   float scale_log2;
 };
 
@@ -343,7 +343,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(BAR_FULL + s), 1); mbar_init(bar(BAR_EMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(BAR_TFULL + i), 1); mbar_init(bar(BAR_TEMPTY + i), 4);
+      mbar_init(bar(BAR_TFULL + i), 1); mbar_init(bar(BAR_TEMPTY + i), 8);
       mbar_init(bar(BAR_QFULL + i), 1); mbar_init(bar(BAR_QEMPTY + i), 1);
     }
     mbar_init(bar(BAR_DRAIN), 1);
@@ -536,10 +536,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
   } else {
     // =============================== epilogue ===================================
-    const int set = (warp - 4) >> 2;    // tiles item%2 == set, accumulator `set`
+    // 16 warps: set = which accumulator (tiles item%2 == set); within a set two warps share each
+    // TMEM lane quarter and split the accumulator's columns in halves (`sub`).
+    const int e = warp - 4;
+    const int set = e >> 3, sub = (e >> 2) & 1;
     const int quarter = warp & 3;       // TMEM lanes 32*quarter .. +31 are this warp's
-    const int st = quarter * 32 + lane;                        // thread of the set, 0..127
-    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 256);
+    const int lt = quarter * 32 + lane;                        // TMEM lane of this thread, 0..127
+    const int st = (e & 7) * 32 + lane;                        // thread of the set, 0..255
+    const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 256);
     const float scale = a.scale_log2;
     const f32x2 scale2 = pk(scale, scale);
     float* negoff = s_negoff + set * 256;
@@ -547,26 +551,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     ItemWalk w(a);
     int item = 0, cur_ph = -1, mine = 0;    // `mine`: tiles this set has taken
     bool dead = false;                      // a wait expired: keep the barrier sequence, skip the work
-    // pass-1 state of rows st and st + 128: sum of 2^(x - mref) over the keys seen so far.  mref is the
+    // pass-1 state of row sub*128 + lt: sum of 2^(x - mref) over the keys seen so far.  mref is the
     // maximum of the first 32 keys the row met; later blocks do not track the maximum (their terms may
     // exceed 1, fp32 has the range), unless a sum overflows, in which case the tile is redone with it.
-    float mref0 = -INFINITY, mref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float mref = -INFINITY, l = 0.f;
     bool first_tile = true;                 // this set has not yet taken a tile of the current pass-1 phase
     for (; w.valid(); w.next(), ++item) {
       const TcPhase p = w.phase();
       if (w.ph != cur_ph) {
         cur_ph = w.ph;
         if (p.pass == 1) {
-          mref0 = mref1 = -INFINITY;
-          l0 = l1 = 0.f;
+          mref = -INFINITY;
+          l = 0.f;
           first_tile = true;
         } else {
           // the segment's offsets: wait until every row has been folded, then stage -offset for this set
           if (!dead) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
-          bar_sync(2 + set, 128);                                 // the set is done with the previous offsets
+          bar_sync(2 + set, 256);                                 // the set is done with the previous offsets
           const float* off = a.offsets + (int64_t)p.seg * NC;
-          for (int i = st; i < NC; i += 128) negoff[i] = dead ? 0.f : -__ldcg(off + i);
-          bar_sync(2 + set, 128);
+          if (st < NC) negoff[st] = dead ? 0.f : -__ldcg(off + st);
+          bar_sync(2 + set, 256);
         }
       }
       if ((item & 1) == set) {
@@ -578,142 +582,110 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!dead) {
           tc_fence_after();
           const int tile = w.g - p.g0;
-          // The accumulator is read 32 columns at a time into two register buffers: the load of
-          // block i+1 is in flight while block i is processed.  The loop over blocks stays rolled
-          // (two blocks per trip) so that the code fits the instruction cache.
-          uint32_t b0[32], b1[32];
-          auto release = [&]() {                                   // accumulator fully read: hand it back
+          uint32_t cur[32];
+          auto release = [&]() {                                   // this warp has read its part of the accumulator
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + set));
           };
           if (p.pass == 1) {
-            // ---- pass 1: sum of 2^(x - mref) of this thread's rows over the tile's 128 keys ----
+            // ---- pass 1: sum of 2^(x - mref) of this thread's row over the tile's 128 keys ----
             // Fast walk: every key of the tile is visible to every row; it does not track the maximum.
             // Careful walk (tiles that reach into the window, or after a sum overflowed in the fast
-            // walk): per-row masks, block maxima, MUFU only.  The two walks are separate loops so that the rare one costs the
-            // common one nothing.
-            const int nblk = 4 * nhalf;
-            const float keep_m0 = mref0, keep_m1 = mref1, keep_l0 = l0, keep_l1 = l1;
-            bool careful = tile * KT + KT - 1 > p.T;
-            if (!careful) {
-              auto block1 = [&](const uint32_t(&cur)[32], int blk) {
-                const bool hf = blk >= 4;
-                if (first_tile && (blk & 3) == 0) {               // first block of these rows: its maximum is the reference
-                  float c0 = fmaxf(__uint_as_float(cur[0]), __uint_as_float(cur[1]));
-                  float c1 = fmaxf(__uint_as_float(cur[2]), __uint_as_float(cur[3]));
-#pragma unroll
-                  for (int i = 4; i < 32; i += 4) {
-                    c0 = fmaxf(c0, fmaxf(__uint_as_float(cur[i]), __uint_as_float(cur[i + 1])));
-                    c1 = fmaxf(c1, fmaxf(__uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3])));
-                  }
-                  if (hf) mref1 = fmaxf(c0, c1) * scale; else mref0 = fmaxf(c0, c1) * scale;
-                }
-                const float mr = hf ? mref1 : mref0;
-                const f32x2 nm2 = pk(-mr, -mr);
-                const float bs = exp_sum32(cur, scale2, [&](int) { return nm2; });
-                if (hf) l1 += bs; else l0 += bs;
-              };
-              tc_ld32_issue(lane_addr, b0);
-              tc_ld_wait(b0);
+            // walk): per-row masks, block maxima, MUFU only.
+            if (sub < nhalf) {
+              const uint32_t addr = lane_base + (uint32_t)(sub * 128);
+              const float keep_m = mref, keep_l = l;
+              bool careful = tile * KT + KT - 1 > p.T;
+              if (!careful) {
 #pragma unroll 1
-              for (int blk = 0; blk < nblk; blk += 2) {
-                tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
-                block1(b0, blk);
-                tc_ld_wait(b1);
-                const bool more = blk + 2 < nblk;
-                if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
-                block1(b1, blk + 1);
-                if (more) tc_ld_wait(b0);
+                for (int blk = 0; blk < 4; ++blk) {
+                  tc_ld32_issue(addr + (uint32_t)(blk * 32), cur);
+                  tc_ld_wait(cur);
+                  if (first_tile && blk == 0) {                    // first block of the row: its maximum is the reference
+                    float c0 = fmaxf(__uint_as_float(cur[0]), __uint_as_float(cur[1]));
+                    float c1 = fmaxf(__uint_as_float(cur[2]), __uint_as_float(cur[3]));
+#pragma unroll
+                    for (int i = 4; i < 32; i += 4) {
+                      c0 = fmaxf(c0, fmaxf(__uint_as_float(cur[i]), __uint_as_float(cur[i + 1])));
+                      c1 = fmaxf(c1, fmaxf(__uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3])));
+                    }
+                    mref = fmaxf(c0, c1) * scale;
+                  }
+                  const f32x2 nm2 = pk(-mref, -mref);
+                  l += exp_sum32(cur, scale2, [&](int) { return nm2; });
+                }
+                // a term beyond fp32 range (a logit 127 above the reference): redo the tile carefully
+                careful = __any_sync(0xffffffffu, !(l < INFINITY));
+                if (careful) { mref = keep_m; l = keep_l; }
               }
-              // a term beyond fp32 range (a logit 127 above the reference): redo the tile carefully
-              careful = __any_sync(0xffffffffu, !(l0 < INFINITY) || !(l1 < INFINITY));
-              if (careful) { mref0 = keep_m0; mref1 = keep_m1; l0 = keep_l0; l1 = keep_l1; }
-            }
-            if (careful) {
-              auto block1c = [&](const uint32_t(&cur)[32], int blk) {
-                const bool hf = blk >= 4;
-                const int j0 = tile * KT + (blk & 3) * 32;
-                const int row = (hf ? 128 : 0) + st;
+              if (careful) {
+                const int row = sub * 128 + lt;
                 const int lastkey = p.T + (p.chunk * NC + row) % a.W;       // last key this row sees
-                if (j0 <= lastkey) {
-                  float mr = hf ? mref1 : mref0;
-                  float ls = hf ? l1 : l0;
-                  float c = -INFINITY;
-#pragma unroll
-                  for (int i = 0; i < 32; ++i) c = fmaxf(c, (j0 + i <= lastkey) ? __uint_as_float(cur[i]) : -INFINITY);
-                  const float mn = fmaxf(mr, c * scale);
-                  float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                  for (int i = 0; i < 32; i += 2) {
-                    s0 += (j0 + i <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i]), scale, -mn)) : 0.f;
-                    s1 += (j0 + i + 1 <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -mn)) : 0.f;
-                  }
-                  ls = fmaf(ls, ex2(mr - mn), s0 + s1);
-                  if (hf) { mref1 = mn; l1 = ls; } else { mref0 = mn; l0 = ls; }
-                }
-              };
 #pragma unroll 1
-              for (int blk = 0; blk < nblk; ++blk) {
-                tc_ld32_issue(lane_addr + (uint32_t)(blk * 32), b0);
-                tc_ld_wait(b0);
-                block1c(b0, blk);
+                for (int blk = 0; blk < 4; ++blk) {
+                  tc_ld32_issue(addr + (uint32_t)(blk * 32), cur);
+                  tc_ld_wait(cur);
+                  const int j0 = tile * KT + blk * 32;
+                  if (j0 <= lastkey) {
+                    float c = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) c = fmaxf(c, (j0 + i <= lastkey) ? __uint_as_float(cur[i]) : -INFINITY);
+                    const float mn = fmaxf(mref, c * scale);
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                      s0 += (j0 + i <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i]), scale, -mn)) : 0.f;
+                      s1 += (j0 + i + 1 <= lastkey) ? ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -mn)) : 0.f;
+                    }
+                    l = fmaf(l, ex2(mref - mn), s0 + s1);
+                    mref = mn;
+                  }
+                }
               }
+              if (l > 0x1p60f) { l *= 0x1p-60f; mref += 60.f; }     // exact: keeps the running sum far from overflow
             }
             release();
-            // exact rescaling keeps the running sums far from overflow
-            if (l0 > 0x1p60f) { l0 *= 0x1p-60f; mref0 += 60.f; }
-            if (l1 > 0x1p60f) { l1 *= 0x1p-60f; mref1 += 60.f; }
             first_tile = false;
           } else {
-            // ---- pass 2: this thread's key, exp2(x - offset[row]) summed over the chunk's rows ----
-            const int nblk = NC >> 5;
-            float sums[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) sums[q] = 0.f;
-            auto block2 = [&](const uint32_t(&cur)[32], int blk) {
-              const float4* no = reinterpret_cast<const float4*>(negoff + blk * 32);
-              float4 o[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) o[i] = no[i];
+            // ---- pass 2: this thread's key, exp2(x - offset[row]) summed over its half of the chunk's rows ----
+            const int half_cols = NC >> 1, nblk = half_cols >> 5;
+            const uint32_t addr = lane_base + (uint32_t)(sub * half_cols);
+            const float* no_base = negoff + sub * half_cols;
+            float sums[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+            for (int blk = 0; blk < nblk; ++blk) {
+              tc_ld32_issue(addr + (uint32_t)(blk * 32), cur);
+              tc_ld_wait(cur);
+              if (blk + 1 == nblk) release();
+              const float2* no = reinterpret_cast<const float2*>(no_base + blk * 32);
               const float bs = exp_sum32(cur, scale2, [&](int pi) {
-                const float4 v = o[pi >> 1];
-                return (pi & 1) ? pk(v.z, v.w) : pk(v.x, v.y);
+                const float2 v = no[pi];
+                return pk(v.x, v.y);
               });
               if (PER_Q) {                                         // W is a multiple of 32: a block never straddles heads
                 const int slot = (blk * 32) / a.W;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) sums[q] += (q == slot) ? bs : 0.f;
+                for (int q = 0; q < 4; ++q) sums[q] += (q == slot) ? bs : 0.f;
               } else {
                 sums[0] += bs;
               }
-            };
-            tc_ld32_issue(lane_addr, b0);
-            tc_ld_wait(b0);
-#pragma unroll 1
-            for (int blk = 0; blk < nblk; blk += 2) {
-              tc_ld32_issue(lane_addr + (uint32_t)((blk + 1) * 32), b1);
-              block2(b0, blk);
-              tc_ld_wait(b1);
-              const bool more = blk + 2 < nblk;
-              if (more) tc_ld32_issue(lane_addr + (uint32_t)((blk + 2) * 32), b0);
-              else release();
-              block2(b1, blk + 1);
-              if (more) tc_ld_wait(b0);
             }
-            const int j = tile * KT + st;
+            const int j = tile * KT + lt;
             if (j < p.T) {
               if (PER_Q) {
-                const int nslot = NC / a.W;
+                // heads of this half: half_cols / W of them, or a part of one head when W > half_cols
+                const int col0 = p.chunk * NC + sub * half_cols;
+                if (a.W > half_cols) {
+                  a.u[(int64_t)((p.h * a.G + col0 / a.W) * 2 + sub) * a.sum_T + p.t_off + j] = sums[0];
+                } else {
+                  const int nslot = half_cols / a.W;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  if (q < nslot) {
-                    const int head = p.h * a.G + (p.chunk * NC) / a.W + q;
-                    a.u[(int64_t)head * a.sum_T + p.t_off + j] = sums[q];
-                  }
+                  for (int q = 0; q < 4; ++q)
+                    if (q < nslot) a.u[(int64_t)((p.h * a.G + col0 / a.W + q) * a.u_parts) * a.sum_T + p.t_off + j] = sums[q];
                 }
               } else {
-                a.u[(int64_t)(p.h * a.u_rows_per_kv + p.chunk) * a.sum_T + p.t_off + j] = sums[0];
+                a.u[(int64_t)(p.h * a.u_rows_per_kv + p.chunk * 2 + sub) * a.sum_T + p.t_off + j] = sums[0];
               }
             }
           }
@@ -722,9 +694,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (w.last_in_phase() && p.pass == 1) {
         // ---- end of a pass-1 phase in this CTA: each set publishes its own (reference, sum) per row ----
         float2* out = a.partials + (((int64_t)p.seg * gridDim.x + blockIdx.x) * 2 + set) * NC;
-        if (st < NC) __stcg(out + st, make_float2(mref0, dead ? 0.f : l0));
-        if (128 + st < NC) __stcg(out + 128 + st, make_float2(mref1, dead ? 0.f : l1));
-        bar_sync(2 + set, 128);
+        const int row = sub * 128 + lt;
+        if (sub < nhalf && row < NC) __stcg(out + row, make_float2(mref, dead ? 0.f : l));
+        bar_sync(2 + set, 256);
         if (st == 0) {                 // the barrier orders the set's stores before this thread's fence: the release is cumulative
           __threadfence();
           atomicAdd(a.published + p.seg, 1u);
@@ -891,6 +863,7 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* 
   a.total_items = tp.total_items;
   a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads;
   a.u_rows_per_kv = c->u_rows_per_kv;
+  a.u_parts = c->u_parts;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.head_dim));
   // every CTA must be resident at once (pass 2 waits for counters other CTAs advance): one CTA per SM at most
   const int grid = tp.grid;
