@@ -120,6 +120,27 @@ def dist_env():
     return rank, world, local
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Requests are sharded by rank with no exchange: each rank draws its own seeded inputs."""
+    return seed + rank
+
+
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """Time of the slowest rank (the only reduction on the multi-GPU path)."""
+    if world == 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank's tokens over the slowest rank's step time."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------------
 def oracle_step(wl, x, layer, controllers, heads=None):
     """One layer of the path by the fp64 oracle (optionally only the first `heads` kv heads)."""
@@ -216,7 +237,7 @@ def run_ours(args):
 
     # resident inputs: a few layers' tensors, rotated (each rank draws its own seed: independent requests)
     n_sets = args.layer_sets
-    host_sets = [I.layer_inputs(wl, l, args.seed + rank) for l in range(n_sets)]
+    host_sets = [I.layer_inputs(wl, l, rank_seed(args.seed, rank)) for l in range(n_sets)]
     pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
     host_pinned = [{k: pin(x[k]) for k in ("q_obs", "k", "v")} for x in host_sets]
     dev_sets = [{k: t.cuda(non_blocking=True).view(torch.bfloat16) for k, t in hp.items()} for hp in host_pinned]
@@ -278,12 +299,9 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     ms_total = t_start.elapsed_time(t_end)
     score_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in score_marks]))
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world)
     ms_step = ms_total / args.steps
-    value = world * wl.total_tokens / (ms_step * 1e-3)
+    value = aggregate_tokens_per_s(wl.total_tokens, world, ms_step)
 
     # ---- per-stage times (serialised, outside the timed region) ----
     marks = []
@@ -321,10 +339,7 @@ def run_ours(args):
         e2e_step(1 + i)
     e1.record(stream)
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / e2e_steps
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / e2e_steps
     h2d = sum(host_pinned[0][k].numel() * 2 for k in ("q_obs", "k", "v"))
     d2h = idx_h.numel() * 4 + ko_h.numel() * 2 + vo_h.numel() * 2 + st_h.numel()
 
@@ -367,7 +382,7 @@ def run_ours(args):
                              f"{work['k_bytes'] / 1e6:.0f} MB per layer",
                        "parallelism": f"replicas x{world}"},
             "roofline": roof, "cpu_baseline": cpu,
-            "e2e": {"value": world * wl.total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": int(launches), "clocks": clocks,
             "stages_ms": {"score+pool": stage_ms[0], "rank_stat": stage_ms[1], "topk": stage_ms[2],
