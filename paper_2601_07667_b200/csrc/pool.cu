@@ -13,51 +13,73 @@
 
 namespace {
 
-__global__ void __launch_bounds__(256) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
-                                                         int Hk, int G, int S, int mode, int urows, int parts, int64_t sum_T,
-                                                         float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
+constexpr int PT = 256;          // tokens per block
+constexpr int MAX_HALO = 16;     // pooling kernels up to 33 taps go through shared memory
+
+// One block pools PT consecutive past tokens of one request.  Row by row, the
+// un-pooled sums of the tile and its halo are staged in shared memory (partial
+// rows added on the way), pooled from there, and added up per kv head and over
+// all heads in a fixed order: no atomics, bit-reproducible.
+__global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
+                                                        int Hk, int G, int S, int mode, int urows, int parts, int64_t sum_T,
+                                                        float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
+  __shared__ float tile[PT + 2 * MAX_HALO];
   const int b = blockIdx.y;
   const AslReq rq = req[b];
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= rq.T) return;
+  const int j0 = blockIdx.x * PT;
+  if (j0 >= rq.T) return;
   const int r = S / 2;
+  const int j = j0 + threadIdx.x;
+  const bool live = j < rq.T;
   const int lo = max(0, j - r), hi = min(rq.T - 1, j + r);
   const float inv = 1.0f / (float)S;
+  // stage sum over `nrows` consecutive rows starting at `row0` for tokens j0-r .. j0+PT-1+r (zero outside [0, T))
+  auto stage = [&](int row0, int nrows) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < PT + 2 * r; i += PT) {
+      const int t = j0 - r + i;
+      float v = 0.f;
+      if (t >= 0 && t < rq.T) {
+        const float* src = u + (int64_t)row0 * sum_T + rq.t_off + t;
+        for (int c = 0; c < nrows; ++c) v += src[(int64_t)c * sum_T];
+      }
+      tile[i] = v;
+    }
+    __syncthreads();
+  };
   float agg = 0.f;
   for (int h = 0; h < Hk; ++h) {
-    float p;
+    float p = 0.f;
     if (mode == ASL_POOL_AVG) {
-      float s = 0.f;
-      for (int c = 0; c < urows; ++c) {
-        const float* row = u + (int64_t)(h * urows + c) * sum_T + rq.t_off;
-        for (int i = lo; i <= hi; ++i) s += row[i];
+      stage(h * urows, urows);
+      if (live) {
+        float s = 0.f;
+        for (int i = lo; i <= hi; ++i) s += tile[i - j0 + r];
+        p = s * inv;
       }
-      p = s * inv;
     } else {
-      p = 0.f;
       for (int g = 0; g < G; ++g) {
-        const float* row = u + (int64_t)(h * G + g) * parts * sum_T + rq.t_off;
-        float mx = -INFINITY;
-        for (int i = lo; i <= hi; ++i) {
-          float v = row[i];
-          for (int c = 1; c < parts; ++c) v += row[(int64_t)c * sum_T + i];     // partial sums of one head come first
-          mx = fmaxf(mx, v);
+        stage((h * G + g) * parts, parts);
+        if (live) {
+          float mx = tile[lo - j0 + r];
+          for (int i = lo + 1; i <= hi; ++i) mx = fmaxf(mx, tile[i - j0 + r]);
+          p += mx;
         }
-        p += mx;
       }
     }
-    scores_kv[(int64_t)h * sum_T + rq.t_off + j] = p;
+    if (live) scores_kv[(int64_t)h * sum_T + rq.t_off + j] = p;
     agg += p;
   }
-  scores_agg[rq.t_off + j] = agg;
+  if (live) scores_agg[rq.t_off + j] = agg;
 }
 
 }  // namespace
 
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st) {
   const asl_params& p = c->p;
-  dim3 grid((c->max_T + 255) / 256, p.batch);
-  pool_group_kernel<<<grid, 256, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
+  if (p.pool_kernel / 2 > MAX_HALO) return ASL_ERR_UNSUPPORTED;
+  dim3 grid((c->max_T + PT - 1) / PT, p.batch);
+  pool_group_kernel<<<grid, PT, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
                                           p.pool_mode, c->u_rows_per_kv, c->u_parts, c->sum_T, scores_kv, scores_agg);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
