@@ -232,6 +232,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = make_workload(args)
+    if args.score_ctas < 0:
+        args.score_ctas = max(1, torch.cuda.get_device_properties(local).multi_processor_count + args.score_ctas)
     work = algorithmic_work(wl)
     pk = peaks()
 
@@ -245,7 +247,7 @@ def run_ours(args):
 
     path = B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
                        pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
-                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local)
+                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=args.score_ctas)
 
     def barrier():
         if world > 1:
@@ -380,7 +382,7 @@ def run_ours(args):
                        "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"],
                        "l2": f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
                              f"{work['k_bytes'] / 1e6:.0f} MB per layer",
-                       "parallelism": f"replicas x{world}"},
+                       "score_ctas": args.score_ctas, "parallelism": f"replicas x{world}"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
@@ -403,6 +405,9 @@ def main():
     ap.add_argument("--layer-sets", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--score-ctas", type=int, default=-16,
+                    help="CTAs of the persistent scorer: 0 = one per SM, negative = that many fewer than SMs.  Fewer "
+                         "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")
     ap.add_argument("--seqlens", type=str, default=None,
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")

@@ -69,7 +69,9 @@ typedef struct {
   int32_t batch;          /* B >= 1 requests                                          */
   int32_t l_min;          /* first layer at which the statistic is evaluated          */
   int32_t l_obs;          /* rank rows kept (ring depth), >= 2                        */
-  int32_t reserved;
+  int32_t score_ctas;     /* CTAs of the persistent scorer kernel; 0 = one per SM.  A   */
+                          /* smaller number leaves SMs to kernels of other streams    */
+                          /* (the previous layer's statistic, top-k and compaction)   */
   double tau;             /* selection fires when relative variance < tau             */
   const int32_t* cu_seqlens; /* host [B+1] token offsets, cu_seqlens[0] = 0           */
   const int32_t* budgets;    /* host [B] KV_budget per request, window included       */

@@ -26,7 +26,7 @@ ASL_RANK_STATIC_MAX_T = 262144
 class AslParams(C.Structure):
     _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("window", C.c_int32), ("pool_kernel", C.c_int32), ("pool_mode", C.c_int32),
-                ("batch", C.c_int32), ("l_min", C.c_int32), ("l_obs", C.c_int32), ("reserved", C.c_int32),
+                ("batch", C.c_int32), ("l_min", C.c_int32), ("l_obs", C.c_int32), ("score_ctas", C.c_int32),
                 ("tau", C.c_double),
                 ("cu_seqlens", C.POINTER(C.c_int32)), ("budgets", C.POINTER(C.c_int32)),
                 ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 2), ("v_stride", C.c_int64 * 2)]
@@ -124,10 +124,11 @@ def asl_destroy(ctx: int) -> None:
 
 def asl_plan(ctx: int, *, n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, pool_kernel: int,
              pool_mode: int, cu_seqlens: Sequence[int], budgets: Sequence[int], l_min: int, l_obs: int,
-             tau: float, q_stride: Sequence[int], k_stride: Sequence[int], v_stride: Sequence[int]) -> int:
+             tau: float, q_stride: Sequence[int], k_stride: Sequence[int], v_stride: Sequence[int],
+             score_ctas: int = 0) -> int:
     cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
     bu = (C.c_int32 * len(budgets))(*[int(x) for x in budgets])
-    p = AslParams(n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, len(budgets), l_min, l_obs, 0,
+    p = AslParams(n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, len(budgets), l_min, l_obs, int(score_ctas),
                   float(tau), cu, bu, (C.c_int64 * 3)(*q_stride), (C.c_int64 * 2)(*k_stride),
                   (C.c_int64 * 2)(*v_stride))
     if len(cu_seqlens) != len(budgets) + 1:
@@ -188,14 +189,17 @@ def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
 class LayerPath:
     """Owns a context, its plan and the device buffers of one layer's pass
     (scores, indices, compacted cache, rank ring, statistic), all torch tensors.
-    ``run_layer`` issues the five steps; the rank statistic goes to a side stream
-    and is not waited for: it overlaps the top-k and the compaction of its own
-    layer and the scoring of the next one (the aggregate scores are double
-    buffered for that).  ``join`` makes the current stream wait for it;
-    ``read_stat`` joins by itself.  A device-wide synchronize covers it too."""
+    ``run_layer`` issues the five steps: the scoring on the current stream, the
+    rest of the layer (rank statistic, top-k, compaction) on a side stream that
+    is not waited for, so that it overlaps the scoring of the next layer (both
+    score buffers are double buffered for that; give the plan ``score_ctas``
+    below the SM count to leave those kernels somewhere to run).  ``join`` makes
+    the current stream wait for everything issued so far; ``read_stat`` joins by
+    itself.  A device-wide synchronize covers it too."""
 
     def __init__(self, *, n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, seqlens, budgets,
-                 l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None):
+                 l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None,
+                 score_ctas: int = 0):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda", device)
@@ -212,16 +216,16 @@ class LayerPath:
         self.ws_bytes = asl_plan(self.ctx, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
                                  window=window, pool_kernel=pool_kernel, pool_mode=pool_mode, cu_seqlens=cu,
                                  budgets=budgets, l_min=l_min, l_obs=l_obs, tau=tau, q_stride=q_stride,
-                                 k_stride=k_stride, v_stride=v_stride)
+                                 k_stride=k_stride, v_stride=v_stride, score_ctas=score_ctas)
         self.sum_tokens, self.sum_T, self.sum_kept = asl_plan_sizes(self.ctx)
         self.kept = [min(int(bg), n) for bg, n in zip(budgets, self.seqlens)]
         self.t_off = np.concatenate([[0], np.cumsum([n - window for n in self.seqlens])]).astype(np.int64)
         self.kept_off = np.concatenate([[0], np.cumsum(self.kept)]).astype(np.int64)
         dev = self.dev
         self.workspace = torch.empty(max(self.ws_bytes, 256), dtype=torch.uint8, device=dev)
-        self.scores_kv = torch.empty((n_kv_heads, self.sum_T), dtype=torch.float32, device=dev)
+        self._kv = [torch.empty((n_kv_heads, self.sum_T), dtype=torch.float32, device=dev) for _ in range(2)]
         self._agg = [torch.empty((self.sum_T,), dtype=torch.float32, device=dev) for _ in range(2)]
-        self._agg_free = [None, None]       # event after the statistic that last read the buffer
+        self._agg_free = [None, None]       # event after the side-stream work that last read the buffers
         self._cur = 0
         self.idx = torch.empty((n_kv_heads, self.sum_kept), dtype=torch.int32, device=dev)
         self.k_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
@@ -232,6 +236,11 @@ class LayerPath:
         self._fork = torch.cuda.Event()
         self._join = torch.cuda.Event()
         self.first_layer: Optional[int] = None
+
+    @property
+    def scores_kv(self):
+        """Per-kv-head scores of the latest layer (device fp32 [H_k][sum_T])."""
+        return self._kv[self._cur]
 
     @property
     def scores_agg(self):
@@ -272,28 +281,28 @@ class LayerPath:
         rows = self.n_rows(layer_idx)
         main = torch.cuda.current_stream()
         self._cur ^= 1
-        agg = self._agg[self._cur]
+        agg, skv = self._agg[self._cur], self._kv[self._cur]
         if self._agg_free[self._cur] is not None:
-            main.wait_event(self._agg_free[self._cur])      # the statistic of two layers ago has read it
+            main.wait_event(self._agg_free[self._cur])      # the side work of two layers ago has read them
         if score_marks is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(main)
-        asl_score_layer(ctx, q_obs, k, self.scores_kv, agg, ws, wsb)
+        asl_score_layer(ctx, q_obs, k, skv, agg, ws, wsb)
         if score_marks is not None:
             e1.record(main)
             score_marks.append((e0, e1))
+        tail = self.side if overlap else main
         if overlap:
             self._fork.record(main)
             self.side.wait_event(self._fork)
-            asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, self.side)
+        asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, tail)
+        asl_select_topk(ctx, skv, self.H_k, self.idx, ws, wsb, tail)
+        asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out, tail)
+        if overlap:
             done = torch.cuda.Event()
             done.record(self.side)
             self._agg_free[self._cur] = done
             self._join.record(self.side)
-        else:
-            asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb)
-        asl_select_topk(ctx, self.scores_kv, self.H_k, self.idx, ws, wsb)
-        asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out)
 
     def read_stat(self) -> np.ndarray:
         """Device -> host copy of the [B] statistic records (synchronises)."""

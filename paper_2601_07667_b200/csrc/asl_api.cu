@@ -63,7 +63,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   if (p->window < 1 || p->batch < 1) return ASL_ERR_INVALID;
   if (p->pool_kernel < 1 || p->pool_kernel % 2 == 0) return ASL_ERR_INVALID;
   if (p->pool_mode != ASL_POOL_AVG && p->pool_mode != ASL_POOL_MAX) return ASL_ERR_INVALID;
-  if (p->l_obs < 2 || p->l_min < 0) return ASL_ERR_INVALID;
+  if (p->l_obs < 2 || p->l_min < 0 || p->score_ctas < 0) return ASL_ERR_INVALID;
   if (p->head_dim < 8 || p->head_dim % 8) return ASL_ERR_INVALID;
   if (p->head_dim != 128) return ASL_ERR_UNSUPPORTED;
   // rows must start on 16-byte boundaries: every stride a multiple of 8 elements

@@ -756,7 +756,7 @@ bool asl_tc_plan(asl_ctx* c) {
   if (NC < 64 || NC % 64 || R % NC) return false;
   tp.NC = NC;
   tp.nchunk = R / NC;
-  tp.grid = c->sm_count;
+  tp.grid = (p.score_ctas > 0 && p.score_ctas < c->sm_count) ? p.score_ctas : c->sm_count;
 
   // segments in (request, head, chunk) order; phases in groups: pass 1 of `group` segments, then their pass 2
   struct Seg { int b, h, chunk, tiles1, tiles2; };
