@@ -158,7 +158,7 @@ asl_status asl_compact_kv(asl_ctx* ctx, const void* k, const void* v, const int3
  * Such a caller can use neither asl_create/asl_plan (both allocate small device
  * tables) nor a workspace it has nowhere to take from.  This call needs no
  * context and no workspace: its sort scratch is a fixed array compiled into
- * the library (about 4.1 MiB of device memory on every GPU that loads the
+ * the library (about 4.2 MiB of device memory on every GPU that loads the
  * library, held until the process exits).
  *
  *   scores    device fp32 [T]   one request's aggregate scores
