@@ -123,6 +123,18 @@ asl_status asl_plan_sizes(const asl_ctx* ctx, int64_t* sum_tokens, int64_t* sum_
 asl_status asl_score_layer(asl_ctx* ctx, const void* q_obs, const void* k, float* scores_kv,
                            float* scores_agg, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same scores when the caller already holds the softmax denominators of the
+ * window rows (Algorithm 1 line 3 is a softmax: A = exp(s - lse) with
+ * lse = log sum over the visible keys of exp(s), s = q.k/sqrt(d); a fused
+ * attention forward keeps exactly this value per query row).  One pass over K
+ * instead of two.  lse: device fp32 [B][H_q][W], natural logarithm. */
+asl_status asl_score_layer_lse(asl_ctx* ctx, const void* q_obs, const void* k, const float* lse, float* scores_kv,
+                               float* scores_agg, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Denominators found by the latest asl_score_layer call on this workspace, in
+ * the layout asl_score_layer_lse takes: lse_out device fp32 [B][H_q][W]. */
+asl_status asl_window_lse(asl_ctx* ctx, const void* workspace, size_t workspace_bytes, float* lse_out, void* stream);
+
 /* Algorithm 1 line 9 + Algorithm 2: writes rank row RankDesc(scores_agg)
  * (0-based, ties to the lower index) into ring slot layer_idx % L_obs of
  * rank_ring (device int32 [L_obs][sum_T]), then, if layer_idx >= L_min and

@@ -66,6 +66,23 @@ def window_attention(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
     return e / e.sum(axis=1, keepdims=True)
 
 
+def window_lse(q_obs: np.ndarray, k: np.ndarray, group: int) -> np.ndarray:
+    """lse[a][t] = log of the softmax denominator of window row t of query head a:
+    log sum over the visible keys j <= n-w+t of exp(q.k_j / sqrt(d)) (Alg. 1 line 3;
+    the quantity a fused attention forward keeps per row).  Returns [H_q][w]."""
+    Hq, w, d = q_obs.shape
+    n = k.shape[0]
+    T = n - w
+    out = np.empty((Hq, w), dtype=np.float64)
+    for a in range(Hq):
+        s = (q_obs[a] @ k[:, a // group, :].T) / math.sqrt(d)
+        for t in range(w):
+            row = s[t, :T + t + 1]
+            m = row.max()
+            out[a, t] = m + math.log(np.exp(row - m).sum())
+    return out
+
+
 def past_column_sums(q_obs: np.ndarray, k: np.ndarray, group: int,
                      return_window_mass: bool = False):
     """U[a][j] = sum_t A[a][t][j] for past columns j < n-w (Alg. 1 line 4).

@@ -19,7 +19,7 @@ ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
-           "asl_rank_desc_static")
+           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -62,6 +62,8 @@ def _load() -> C.CDLL:
     lib.asl_plan.argtypes = [vp, C.POINTER(AslParams), C.POINTER(sz)]
     lib.asl_plan_sizes.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
     lib.asl_score_layer.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.asl_score_layer_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.asl_window_lse.argtypes = [vp, vp, sz, vp, vp]
     lib.asl_rank_stat.argtypes = [vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.asl_select_topk.argtypes = [vp, vp, i32, vp, vp, sz, vp]
     lib.asl_compact_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -149,6 +151,16 @@ def asl_score_layer(ctx, q_obs, k, scores_kv, scores_agg, workspace, workspace_b
                                 int(workspace_bytes), _stream_handle(stream)), "asl_score_layer")
 
 
+def asl_score_layer_lse(ctx, q_obs, k, lse, scores_kv, scores_agg, workspace, workspace_bytes, stream=None) -> None:
+    _check(_lib.asl_score_layer_lse(ctx, _ptr(q_obs), _ptr(k), _ptr(lse), _ptr(scores_kv), _ptr(scores_agg),
+                                    _ptr(workspace), int(workspace_bytes), _stream_handle(stream)), "asl_score_layer_lse")
+
+
+def asl_window_lse(ctx, workspace, workspace_bytes, lse_out, stream=None) -> None:
+    _check(_lib.asl_window_lse(ctx, _ptr(workspace), int(workspace_bytes), _ptr(lse_out), _stream_handle(stream)),
+           "asl_window_lse")
+
+
 def asl_rank_stat(ctx, scores_agg, layer_idx, n_rows, rank_ring, stat, workspace, workspace_bytes, stream=None) -> None:
     _check(_lib.asl_rank_stat(ctx, _ptr(scores_agg), int(layer_idx), int(n_rows), _ptr(rank_ring), _ptr(stat),
                               _ptr(workspace), int(workspace_bytes), _stream_handle(stream)), "asl_rank_stat")
@@ -182,7 +194,7 @@ def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
     shared by every call on the device, so calls that could overlap on the GPU
     must be ordered; T is limited to ASL_RANK_STATIC_MAX_T."""
     _check(_lib.asl_rank_desc_static(_ptr(scores), int(T), _ptr(rank_out), _stream_handle(stream)),
-           "asl_rank_desc_static")
+           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse")
 
 
 # ---- a small holder of one plan's device buffers -------------------------------------
@@ -272,7 +284,7 @@ class LayerPath:
             self.first_layer = layer_idx
         return min(self.l_obs, layer_idx - self.first_layer + 1)
 
-    def run_layer(self, q_obs, k, v, layer_idx: int, *, overlap: bool = True, score_marks=None) -> None:
+    def run_layer(self, q_obs, k, v, layer_idx: int, *, overlap: bool = True, score_marks=None, lse=None) -> None:
         """Steps a1..a5 for one layer on the current stream; with ``overlap`` the statistic
         runs on the side stream and is left in flight (see ``join``).  ``score_marks``: a list
         that receives a (start, end) event pair around the scoring call."""
@@ -287,7 +299,10 @@ class LayerPath:
         if score_marks is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(main)
-        asl_score_layer(ctx, q_obs, k, skv, agg, ws, wsb)
+        if lse is None:
+            asl_score_layer(ctx, q_obs, k, skv, agg, ws, wsb)
+        else:                                               # the caller holds the window rows' log-sum-exp: one pass
+            asl_score_layer_lse(ctx, q_obs, k, lse, skv, agg, ws, wsb)
         if score_marks is not None:
             e1.record(main)
             score_marks.append((e0, e1))

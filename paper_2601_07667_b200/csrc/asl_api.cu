@@ -165,16 +165,33 @@ asl_status asl_plan_sizes(const asl_ctx* c, int64_t* sum_tokens, int64_t* sum_T,
   return ASL_OK;
 }
 
-asl_status asl_score_layer(asl_ctx* c, const void* q_obs, const void* k, float* scores_kv, float* scores_agg,
-                           void* workspace, size_t workspace_bytes, void* stream) {
+static asl_status score_layer_impl(asl_ctx* c, const void* q_obs, const void* k, const float* lse, float* scores_kv,
+                                   float* scores_agg, void* workspace, size_t workspace_bytes, void* stream) {
   if (!c || !c->planned || !q_obs || !k || !scores_kv || !scores_agg) return ASL_ERR_INVALID;
   if (!aligned16(q_obs) || !aligned16(k)) return ASL_ERR_INVALID;
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
   if (c->tc.enabled && !c->force_simt)
-    return asl_launch_score_tc(c, q_obs, k, scores_kv, scores_agg, static_cast<char*>(workspace),
+    return asl_launch_score_tc(c, q_obs, k, lse, scores_kv, scores_agg, static_cast<char*>(workspace),
                                static_cast<cudaStream_t>(stream));
-  return asl_launch_score_simt(c, q_obs, k, scores_kv, scores_agg, static_cast<char*>(workspace),
+  return asl_launch_score_simt(c, q_obs, k, lse, scores_kv, scores_agg, static_cast<char*>(workspace),
                                static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_score_layer(asl_ctx* c, const void* q_obs, const void* k, float* scores_kv, float* scores_agg,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  return score_layer_impl(c, q_obs, k, nullptr, scores_kv, scores_agg, workspace, workspace_bytes, stream);
+}
+
+asl_status asl_score_layer_lse(asl_ctx* c, const void* q_obs, const void* k, const float* lse, float* scores_kv,
+                               float* scores_agg, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!lse) return ASL_ERR_INVALID;
+  return score_layer_impl(c, q_obs, k, lse, scores_kv, scores_agg, workspace, workspace_bytes, stream);
+}
+
+asl_status asl_window_lse(asl_ctx* c, const void* workspace, size_t workspace_bytes, float* lse_out, void* stream) {
+  if (!c || !c->planned || !lse_out) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  return asl_launch_window_lse(c, static_cast<const char*>(workspace), lse_out, static_cast<cudaStream_t>(stream));
 }
 
 asl_status asl_rank_stat(asl_ctx* c, const float* scores_agg, int32_t layer_idx, int32_t n_rows, int32_t* rank_ring,

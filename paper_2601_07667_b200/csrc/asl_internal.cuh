@@ -68,14 +68,15 @@ struct asl_ctx {
 static inline size_t asl_align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 // ---- kernels' host launchers (one per translation unit) ----
-asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
-                                 char* ws, cudaStream_t st);
+asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
+                                 float* scores_agg, char* ws, cudaStream_t st);
+asl_status asl_launch_window_lse(asl_ctx* c, const char* ws, float* lse_out, cudaStream_t st);
 bool asl_tc_plan(asl_ctx* c);
 void asl_tc_free(asl_ctx* c);
 size_t asl_tc_partial_bytes(const asl_ctx* c);
 asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st);
-asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
-                               char* ws, cudaStream_t st);
+asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
+                               float* scores_agg, char* ws, cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);

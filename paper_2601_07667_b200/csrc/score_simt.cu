@@ -165,10 +165,30 @@ __global__ void __launch_bounds__(128) score_pass2_simt(ScoreArgs a, const float
   }
 }
 
+// offsets[b][h][r] (log2 domain, row r = g*W + t of kv head h) <-> lse[b][h*G + g][t] (natural log)
+__global__ void lse_to_offsets(const float* __restrict__ lse, float* __restrict__ offsets, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) offsets[i] = lse[i] * 1.4426950408889634f;
+}
+__global__ void offsets_to_lse(const float* __restrict__ offsets, float* __restrict__ lse, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) lse[i] = __ldcg(offsets + i) * 0.6931471805599453f;
+}
+
 }  // namespace
 
-asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg,
-                                 char* ws, cudaStream_t st) {
+// The row offsets of the latest asl_score_layer call, as natural-log softmax denominators.
+// [b][h][g*W + t] and [b][h*G + g][t] are the same linear order: contiguous groups.
+asl_status asl_launch_window_lse(asl_ctx* c, const char* ws, float* lse_out, cudaStream_t st) {
+  const int n = c->p.batch * c->p.n_kv_heads * c->rows_per_kv;
+  offsets_to_lse<<<(n + 255) / 256, 256, 0, st>>>(reinterpret_cast<const float*>(ws + c->ws.score_offsets), lse_out, n);
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}
+
+asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
+                                 float* scores_agg, char* ws, cudaStream_t st) {
   const asl_params& p = c->p;
   ScoreArgs a;
   a.q = static_cast<const uint16_t*>(q);
@@ -181,13 +201,20 @@ asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, float
   float2* partials = reinterpret_cast<float2*>(ws + c->ws.score_partials);
   float* offsets = reinterpret_cast<float*>(ws + c->ws.score_offsets);
   float* u = reinterpret_cast<float*>(ws + c->ws.score_u);
-  const int max_tiles = (c->max_n + KT - 1) / KT;
-  dim3 g1(max_tiles, p.n_kv_heads, p.batch);
-  score_pass1_simt<<<g1, 256, 0, st>>>(a, partials);
-  score_combine_simt<<<dim3(p.n_kv_heads, p.batch), 256, 0, st>>>(partials, c->d_req, a.Hk, a.R, offsets);
+  if (lse) {                                    // supplied denominators: pass 2 alone
+    const int n = p.batch * p.n_kv_heads * c->rows_per_kv;
+    lse_to_offsets<<<(n + 255) / 256, 256, 0, st>>>(lse, offsets, n);
+    c->launches += 1;
+  } else {
+    const int max_tiles = (c->max_n + KT - 1) / KT;
+    dim3 g1(max_tiles, p.n_kv_heads, p.batch);
+    score_pass1_simt<<<g1, 256, 0, st>>>(a, partials);
+    score_combine_simt<<<dim3(p.n_kv_heads, p.batch), 256, 0, st>>>(partials, c->d_req, a.Hk, a.R, offsets);
+    c->launches += 2;
+  }
   dim3 g2((c->max_T + KT - 1) / KT, p.n_kv_heads, p.batch);
   score_pass2_simt<<<g2, 128, 0, st>>>(a, offsets, p.pool_mode == ASL_POOL_MAX ? 1 : 0, c->sum_T, u);
-  c->launches += 3;
+  c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return asl_launch_pool(c, u, scores_kv, scores_agg, st);
 }

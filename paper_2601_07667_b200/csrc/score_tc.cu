@@ -285,13 +285,14 @@ struct TcArgs {
   const AslReq* req;
   float2* partials;        // pass 1: [segment][CTA][set][NC] (reference, sum) of each epilogue set
   float* offsets;          // [segment][NC], written by the folding warps, read by pass 2
+  const float* lse;        // null, or the rows' natural-log softmax denominators [B][H_q][W]: pass 2 alone
   float* u;                // pass 2 out: column sums
   uint32_t* published;     // [segment] epilogue sets that have published, accumulated over launches
   uint32_t* folded;        // [segment] rows whose offset is written, accumulated over launches
   int32_t* err;
   int64_t sum_T;
   uint32_t epoch;          // launch number, from 1
-  int32_t n_phases, total_items, NC, W, G, Hk, u_rows_per_kv, u_parts;
+  int32_t n_phases, total_items, NC, W, G, Hk, Hq, u_rows_per_kv, u_parts;
   float scale_log2;
 };
 
@@ -566,10 +567,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           first_tile = true;
         } else {
           // the segment's offsets: wait until every row has been folded, then stage -offset for this set
-          if (!dead) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
+          if (!dead && !a.lse) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
           bar_sync(2 + set, 256);                                 // the set is done with the previous offsets
-          const float* off = a.offsets + (int64_t)p.seg * NC;
-          if (st < NC) negoff[st] = dead ? 0.f : -__ldcg(off + st);
+          if (st < NC) {
+            float off;
+            if (a.lse) {                                          // supplied: natural log -> log2 domain
+              const int r = p.chunk * NC + st;                    // row within the kv head: query head r / W, window row r % W
+              off = __ldg(a.lse + ((int64_t)p.b * a.Hq + p.h * a.G + r / a.W) * a.W + r % a.W) * 1.4426950408889634f;
+            } else {
+              off = __ldcg(a.offsets + (int64_t)p.seg * NC + st);
+            }
+            negoff[st] = dead ? 0.f : -off;
+          }
           bar_sync(2 + set, 256);
         }
       }
@@ -787,8 +796,17 @@ bool asl_tc_plan(asl_ctx* c) {
   if (g >= ((int64_t)1 << 31) - tp.grid) return false;
   tp.total_items = (int32_t)g;
 
+  std::vector<TcPhase> only2;
+  int64_t g2 = 0;
+  for (const TcPhase& ph : tp.phases)
+    if (ph.pass == 2) { TcPhase q = ph; q.g0 = (int32_t)g2; g2 += q.ntiles; only2.push_back(q); }
+  tp.n_phases2 = (int32_t)only2.size();
+  tp.total_items2 = (int32_t)g2;
+
   const size_t sync_bytes = 2 * (size_t)tp.nseg * sizeof(uint32_t);
   cudaError_t e = cudaMalloc(&tp.d_phases, tp.phases.size() * sizeof(TcPhase));
+  if (e == cudaSuccess) e = cudaMalloc(&tp.d_phases2, only2.size() * sizeof(TcPhase));
+  if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases2, only2.data(), only2.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&tp.d_sync, sync_bytes);
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases, tp.phases.data(), tp.phases.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(tp.d_sync, 0, sync_bytes);
@@ -809,8 +827,10 @@ size_t asl_tc_partial_bytes(const asl_ctx* c) {
 void asl_tc_free(asl_ctx* c) {
   AslTcPlan& tp = c->tc;
   if (tp.d_phases) cudaFree(tp.d_phases);
+  if (tp.d_phases2) cudaFree(tp.d_phases2);
   if (tp.d_sync) cudaFree(tp.d_sync);
   tp.d_phases = nullptr;
+  tp.d_phases2 = nullptr;
   tp.d_sync = nullptr;
   tp.enabled = false;
 }
@@ -824,8 +844,8 @@ asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st) {
   return ASL_OK;
 }
 
-asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* scores_kv, float* scores_agg, char* ws,
-                               cudaStream_t st) {
+asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
+                               float* scores_agg, char* ws, cudaStream_t st) {
   const asl_params& p = c->p;
   AslTcPlan& tp = c->tc;
   const int W = p.window, G = p.n_q_heads / p.n_kv_heads, NC = tp.NC;
@@ -848,7 +868,8 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* 
     if (rs != ASL_OK) return rs;
   }
   TcArgs a{};
-  a.phases = tp.d_phases;
+  a.phases = lse ? tp.d_phases2 : tp.d_phases;
+  a.lse = lse;
   a.req = c->d_req;
   a.partials = reinterpret_cast<float2*>(ws + c->ws.score_partials);
   a.offsets = reinterpret_cast<float*>(ws + c->ws.score_offsets);
@@ -858,10 +879,10 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, float* 
   a.folded = tp.d_sync + tp.nseg;
   a.err = c->d_err;
   a.sum_T = c->sum_T;
-  a.epoch = ++tp.epoch;
-  a.n_phases = (int32_t)tp.phases.size();
-  a.total_items = tp.total_items;
-  a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads;
+  a.epoch = lse ? tp.epoch : ++tp.epoch;          // the one-pass launch does not touch the counters
+  a.n_phases = lse ? tp.n_phases2 : (int32_t)tp.phases.size();
+  a.total_items = lse ? tp.total_items2 : tp.total_items;
+  a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads; a.Hq = p.n_q_heads;
   a.u_rows_per_kv = c->u_rows_per_kv;
   a.u_parts = c->u_parts;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.head_dim));

@@ -199,3 +199,30 @@ def test_run_twice_is_bitwise_identical():
         path.close()
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("Hq,Hk,w,mode,n", [(32, 8, 64, 0, 3000), (8, 2, 32, 1, 2000), (6, 2, 40, 0, 900)])
+def test_one_pass_scoring_with_supplied_lse(Hq, Hk, w, mode, n):
+    """asl_score_layer_lse fed the oracle's log-sum-exp gives the oracle's scores; asl_window_lse
+    returns the denominators the two-pass call found (tensor-core shapes and the CUDA-core fallback)."""
+    from paper_2601_07667_b200 import binding as B
+    from asl_check import assert_scores_close, oracle_layer
+    wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, pool_mode=mode, seqlens=(n,), budgets=(w + 50,),
+                    layers=1, l_min=1, l_obs=2)
+    x = I.layer_inputs(wl, 0, seed=8)
+    path = make_path(wl)
+    q, k = to_dev(x["q_obs"]), to_dev(x["k"])
+    lse_ref = O.window_lse(O.widen_bf16(x["q_obs"][0]), O.widen_bf16(x["k"]), wl.group)
+    lse_dev = torch.from_numpy(lse_ref.astype(np.float32)).cuda().reshape(1, Hq, w)
+    B.asl_score_layer_lse(path.ctx, q, k, lse_dev, path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
+    torch.cuda.synchronize()
+    P_ref, agg_ref = oracle_layer(wl, x)
+    assert_scores_close(path.scores_kv.cpu().numpy(), P_ref, "one-pass scores_kv")
+    assert_scores_close(path.scores_agg.cpu().numpy(), agg_ref, "one-pass scores_agg")
+    B.asl_score_layer(path.ctx, q, k, path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
+    got = torch.empty((1, Hq, w), dtype=torch.float32, device="cuda")
+    B.asl_window_lse(path.ctx, path.workspace, path.ws_bytes, got)
+    torch.cuda.synchronize()
+    assert np.abs(got.cpu().numpy()[0].astype(np.float64) - lse_ref).max() <= 2e-4     # log domain, absolute
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()

@@ -299,3 +299,30 @@ def test_score_layer_composition_small():
     Pm, _ = O.score_layer(q, k, 2, S, O.POOL_MAX)
     Vm = torch.nn.functional.max_pool1d(t, S, stride=1, padding=S // 2)[0].numpy()
     assert np.allclose(Pm, Vm[0::2] + Vm[1::2], rtol=1e-12)
+
+
+# ------------------------------------------------------------------ window log-sum-exp
+def test_window_lse_closed_form_and_brute_force():
+    g = rng(21)
+    Hq, Hk, w, d, n = 4, 2, 5, 8, 30
+    T = n - w
+    # identical keys: every visible logit equals s, so lse = s + log(number of visible keys)
+    key = g.standard_normal(d)
+    k = np.broadcast_to(key, (n, Hk, d)).copy()
+    q = g.standard_normal((Hq, w, d))
+    lse = O.window_lse(q, k, Hq // Hk)
+    for a in range(Hq):
+        for t in range(w):
+            s = float(q[a, t] @ key) / math.sqrt(d)
+            assert lse[a, t] == pytest.approx(s + math.log(T + t + 1), abs=1e-12)
+    # random keys: pure-Python sums, and the defining property A = exp(s - lse)
+    k = g.standard_normal((n, Hk, d)) * 2.0
+    lse = O.window_lse(q, k, Hq // Hk)
+    for a in range(Hq):
+        A = O.window_attention(q[a], k[:, a // 2, :])
+        for t in range(w):
+            logits = [math.fsum(float(q[a, t, c]) * float(k[j, a // 2, c]) for c in range(d)) / math.sqrt(d)
+                      for j in range(T + t + 1)]
+            brute = math.log(math.fsum(math.exp(x) for x in logits))
+            assert lse[a, t] == pytest.approx(brute, abs=1e-12)
+            assert A[t, 3] == pytest.approx(math.exp(logits[3] - lse[a, t]), rel=1e-12)
