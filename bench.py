@@ -250,7 +250,8 @@ def run_ours(args):
 
     path = B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
                        pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
-                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=args.score_ctas)
+                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=args.score_ctas,
+                       tail_streams=args.tail_streams)
 
     def barrier():
         if world > 1:
@@ -409,7 +410,7 @@ def run_ours(args):
                        "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"],
                        "l2": f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
                              f"{work['k_bytes'] / 1e6:.0f} MB per layer",
-                       "score_ctas": args.score_ctas, "parallelism": f"replicas x{world}"},
+                       "score_ctas": args.score_ctas, "tail_streams": args.tail_streams, "parallelism": f"replicas x{world}"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
@@ -435,6 +436,8 @@ def main():
     ap.add_argument("--layer-sets", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tail-streams", type=int, default=1, choices=[1, 2],
+                    help="side streams for the rest of the layer: 2 = statistic and top-k/compaction side by side")
     ap.add_argument("--score-ctas", type=int, default=-16,
                     help="CTAs of the persistent scorer: 0 = one per SM, negative = that many fewer than SMs.  Fewer "
                          "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")

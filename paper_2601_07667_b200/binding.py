@@ -202,8 +202,8 @@ class LayerPath:
     """Owns a context, its plan and the device buffers of one layer's pass
     (scores, indices, compacted cache, rank ring, statistic), all torch tensors.
     ``run_layer`` issues the five steps: the scoring on the current stream, the
-    rest of the layer (rank statistic, top-k, compaction) on a side stream that
-    is not waited for, so that it overlaps the scoring of the next layer (both
+    rest of the layer on a side stream (``tail_streams=2``: the rank statistic on
+    one, top-k and compaction on another) that is not waited for, so that it overlaps the scoring of the next layer (both
     score buffers are double buffered for that; give the plan ``score_ctas``
     below the SM count to leave those kernels somewhere to run).  ``join`` makes
     the current stream wait for everything issued so far; ``read_stat`` joins by
@@ -211,7 +211,7 @@ class LayerPath:
 
     def __init__(self, *, n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, seqlens, budgets,
                  l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None,
-                 score_ctas: int = 0):
+                 score_ctas: int = 0, tail_streams: int = 1):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda", device)
@@ -244,9 +244,11 @@ class LayerPath:
         self.v_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
         self.rank_ring = torch.zeros((l_obs, self.sum_T), dtype=torch.int32, device=dev)
         self.stat = torch.zeros((self.batch, C.sizeof(AslStat)), dtype=torch.uint8, device=dev)
-        self.side = torch.cuda.Stream(device=dev)
+        self.side = torch.cuda.Stream(device=dev)       # rank statistic
+        self.side2 = torch.cuda.Stream(device=dev) if tail_streams >= 2 else self.side     # top-k and compaction
         self._fork = torch.cuda.Event()
         self._join = torch.cuda.Event()
+        self._join2 = torch.cuda.Event()
         self.first_layer: Optional[int] = None
 
     @property
@@ -261,7 +263,9 @@ class LayerPath:
 
     def join(self) -> None:
         """The current stream waits for the statistic work issued so far."""
-        self.torch.cuda.current_stream().wait_event(self._join)
+        cur = self.torch.cuda.current_stream()
+        cur.wait_event(self._join)
+        cur.wait_event(self._join2)
 
     def close(self) -> None:
         if self.ctx:
@@ -295,7 +299,8 @@ class LayerPath:
         self._cur ^= 1
         agg, skv = self._agg[self._cur], self._kv[self._cur]
         if self._agg_free[self._cur] is not None:
-            main.wait_event(self._agg_free[self._cur])      # the side work of two layers ago has read them
+            for done in self._agg_free[self._cur]:          # the side work of two layers ago has read them
+                main.wait_event(done)
         if score_marks is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(main)
@@ -306,18 +311,21 @@ class LayerPath:
         if score_marks is not None:
             e1.record(main)
             score_marks.append((e0, e1))
-        tail = self.side if overlap else main
         if overlap:
             self._fork.record(main)
             self.side.wait_event(self._fork)
-        asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, tail)
-        asl_select_topk(ctx, skv, self.H_k, self.idx, ws, wsb, tail)
-        asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out, tail)
+            self.side2.wait_event(self._fork)
+        s1, s2 = (self.side, self.side2) if overlap else (main, main)
+        asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, s1)
+        asl_select_topk(ctx, skv, self.H_k, self.idx, ws, wsb, s2)
+        asl_compact_kv(ctx, k, v, self.idx, self.k_out, self.v_out, s2)
         if overlap:
-            done = torch.cuda.Event()
-            done.record(self.side)
-            self._agg_free[self._cur] = done
+            d1, d2 = torch.cuda.Event(), torch.cuda.Event()
+            d1.record(self.side)
+            d2.record(self.side2)
+            self._agg_free[self._cur] = (d1, d2)
             self._join.record(self.side)
+            self._join2.record(self.side2)
 
     def read_stat(self) -> np.ndarray:
         """Device -> host copy of the [B] statistic records (synchronises)."""
