@@ -4,10 +4,12 @@
  * the ranking of context tokens by observation-window attention settles, and
  * prunes the KV cache to a budget.  This library is the per-layer data path:
  *
- *   asl_score_layer   Algorithm 1 lines 3-6 + the "scores" sum of Section 4.1
- *   asl_rank_stat     Algorithm 1 line 9 + Algorithm 2 lines 1-10 (Section 4.1)
- *   asl_select_topk   Algorithm 1 lines 7-8
- *   asl_compact_kv    Algorithm 1 line 10
+ *   asl_score_layer   Algorithm 1: window softmax A, past-only column sum U, 1-D
+ *                     pooling, SumGroups; plus the "scores" sum of Section 4.1
+ *   asl_rank_stat     Algorithm 1: RankDesc; Algorithm 2 up to the threshold test
+ *                     (rank rows R, TopKIndices J, Unique U, RelNormVar; Section 4.1)
+ *   asl_select_topk   Algorithm 1: k, TopK and the window append
+ *   asl_compact_kv    Algorithm 1: the returned K[I], V[I]
  *
  * Conventions
  *   - Every entry point returns an asl_status; nothing throws, aborts or prints.
@@ -113,10 +115,10 @@ asl_status asl_plan(asl_ctx* ctx, const asl_params* params, size_t* workspace_by
  * sum_kept = sum of min(budget_b, n_b). */
 asl_status asl_plan_sizes(const asl_ctx* ctx, int64_t* sum_tokens, int64_t* sum_T, int64_t* sum_kept);
 
-/* Algorithm 1 lines 3-6: A = softmax over all n keys of the last W query rows
+/* Algorithm 1 up to SumGroups: A = softmax over all n keys of the last W query rows
  * (causal mask on the last W x W block), U = column sums over the W rows for
  * past columns, pooled per query head, summed over each GQA group:
- *   scores_kv  device [H_k][sum_T] fp32   P of Algorithm 1 line 6
+ *   scores_kv  device [H_k][sum_T] fp32   P of Algorithm 1 (SumGroups)
  *   scores_agg device [sum_T]      fp32   sum over kv heads (the "scores" of Section 4.1)
  * q_obs device bf16 [B][H_q][W][d] (strides q_stride), k device bf16 packed
  * [sum n_b][H_k][d] (strides k_stride). */
@@ -124,7 +126,7 @@ asl_status asl_score_layer(asl_ctx* ctx, const void* q_obs, const void* k, float
                            float* scores_agg, void* workspace, size_t workspace_bytes, void* stream);
 
 /* The same scores when the caller already holds the softmax denominators of the
- * window rows (Algorithm 1 line 3 is a softmax: A = exp(s - lse) with
+ * window rows (Algorithm 1 (window softmax A) is a softmax: A = exp(s - lse) with
  * lse = log sum over the visible keys of exp(s), s = q.k/sqrt(d); a fused
  * attention forward keeps exactly this value per query row).  One pass over K
  * instead of two.  lse: device fp32 [B][H_q][W], natural logarithm. */
@@ -135,7 +137,7 @@ asl_status asl_score_layer_lse(asl_ctx* ctx, const void* q_obs, const void* k, c
  * the layout asl_score_layer_lse takes: lse_out device fp32 [B][H_q][W]. */
 asl_status asl_window_lse(asl_ctx* ctx, const void* workspace, size_t workspace_bytes, float* lse_out, void* stream);
 
-/* Algorithm 1 line 9 + Algorithm 2: writes rank row RankDesc(scores_agg)
+/* Algorithm 1 (RankDesc) + Algorithm 2: writes rank row RankDesc(scores_agg)
  * (0-based, ties to the lower index) into ring slot layer_idx % L_obs of
  * rank_ring (device int32 [L_obs][sum_T]), then, if layer_idx >= L_min and
  * n_rows >= 2, takes the statistic over the latest n_rows rows (the rows of
@@ -146,7 +148,7 @@ asl_status asl_rank_stat(asl_ctx* ctx, const float* scores_agg, int32_t layer_id
                          int32_t* rank_ring, asl_stat* stat, void* workspace, size_t workspace_bytes,
                          void* stream);
 
-/* Algorithm 1 lines 7-8 per (request, head): the k_b = min(budget_b, n_b) - W
+/* Algorithm 1 (k, TopK and window append) per (request, head): the k_b = min(budget_b, n_b) - W
  * past tokens with the largest score, ties to the lower index, written in
  * ascending index order and followed by the window indices T_b .. n_b-1.
  * scores device [n_heads][sum_T] fp32; idx_out device int32 [n_heads][sum_kept].
@@ -154,14 +156,27 @@ asl_status asl_rank_stat(asl_ctx* ctx, const float* scores_agg, int32_t layer_id
 asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
                            void* workspace, size_t workspace_bytes, void* stream);
 
-/* Algorithm 1 line 10: k_out[h][r][:] = k[cu_seqlens[b] + idx[h][r]][h][:] and
+/* Algorithm 1 (K[I], V[I]): k_out[h][r][:] = k[cu_seqlens[b] + idx[h][r]][h][:] and
  * the same for v, r running over request b's kept segment.
  * k_out, v_out: device bf16 dense [H_k][sum_kept][d]. */
 asl_status asl_compact_kv(asl_ctx* ctx, const void* k, const void* v, const int32_t* idx, void* k_out,
                           void* v_out, void* stream);
 
+/* Algorithm 2 (one-shot selection), the one-shot selection at the selection layer: once
+ * asl_rank_stat reports `selected`, the tokens that go on to the deeper layers
+ * are select_idx = Unique(J_last u I_w): the k tokens with the best aggregate
+ * score of THIS layer plus the window.  That index list is asl_select_topk with
+ * scores = scores_agg and n_heads = 1 (ascending, window appended: already
+ * unique); this call gathers any per-token tensor with it, for example the
+ * hidden states:  out[kept_off_b + r][:] = x[cu_seqlens[b] + idx[kept_off_b + r]][:].
+ *   x    device, packed [sum n_b] rows of row_bytes bytes (multiple of 16, 16-byte aligned)
+ *   idx  device int32 [sum_kept], as written by asl_select_topk(n_heads = 1)
+ *   out  device, [sum_kept] rows of row_bytes bytes */
+asl_status asl_compact_rows(asl_ctx* ctx, const void* x, const int32_t* idx, void* out, int64_t row_bytes,
+                            void* stream);
+
 /* Rank row without any allocation.  (The paper has no counterpart: this is a
- * packaging of Algorithm 1 line 9 for hosts that may not allocate.)
+ * packaging of Algorithm 1 (RankDesc) for hosts that may not allocate.)
  *
  * Who needs it: a caller that cannot obtain device memory at the time it wants
  * a rank row -- an inference server whose memory pool was handed over to its

@@ -17,16 +17,16 @@ brute force with Python sets.
 Readings taken where the paper leaves a choice (each also listed in the
 design notes):
   * softmax runs over all n keys, window keys included under the causal mask
-    of the last w x w block; only past columns [0, n-w) are kept (Alg. 1 l.3-4);
+    of the last w x w block; only past columns [0, n-w) are kept (Alg. 1 (window softmax A, past-only column sum U));
   * pooling is stride 1, pad floor(S/2); average pooling pads with zeros and
-    always divides by S; max pooling looks at in-range taps only (Alg. 1 l.5);
-  * pooling runs per query head, then heads of a GQA group are summed (Alg. 1
-    l.5-6); the rank statistic orders tokens by the sum over all heads (Sec. 4.1);
+    always divides by S; max pooling looks at in-range taps only (Alg. 1 (1-D pooling));
+  * pooling runs per query head, then heads of a GQA group are summed (Alg. 1:
+    pooling, then SumGroups); the rank statistic orders tokens by the sum over all heads (Sec. 4.1);
   * ranks are 0-based, descending score, ties to the lower index (stable);
-  * the statistic uses the latest L_obs rank rows (Alg. 2 l.5), population
+  * the statistic uses the latest L_obs rank rows (Alg. 2 (stacked rank rows R)), population
     variance of raw ranks, mean over the union of per-row top-k sets;
   * top-k ties go to the lower index; kept indices are emitted ascending with
-    the window indices appended (Alg. 1 l.7-8).
+    the window indices appended (Alg. 1 (k, TopK and window append)).
 """
 from __future__ import annotations
 
@@ -46,11 +46,11 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# Algorithm 1, lines 3-4: window softmax and the past-only column sum U
+# Algorithm 1: window softmax A and the past-only column sum U
 # --------------------------------------------------------------------------
 def window_attention(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
     """A = Softmax(Q[n-w:n] K^T / sqrt(d) + CausalMaskOnLastBlock(w)) for one
-    query head (Alg. 1 line 3; Sec. 4.1 "PA").
+    query head (Alg. 1 (window softmax A); Sec. 4.1 "PA").
 
     q_head [w][d], k_head [n][d], float64.  Row t sits at position n-w+t and
     sees keys j <= n-w+t.  Returns A [w][n]."""
@@ -68,7 +68,7 @@ def window_attention(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
 
 def window_lse(q_obs: np.ndarray, k: np.ndarray, group: int) -> np.ndarray:
     """lse[a][t] = log of the softmax denominator of window row t of query head a:
-    log sum over the visible keys j <= n-w+t of exp(q.k_j / sqrt(d)) (Alg. 1 line 3;
+    log sum over the visible keys j <= n-w+t of exp(q.k_j / sqrt(d)) (Alg. 1 (window softmax A);
     the quantity a fused attention forward keeps per row).  Returns [H_q][w]."""
     Hq, w, d = q_obs.shape
     n = k.shape[0]
@@ -85,10 +85,10 @@ def window_lse(q_obs: np.ndarray, k: np.ndarray, group: int) -> np.ndarray:
 
 def past_column_sums(q_obs: np.ndarray, k: np.ndarray, group: int,
                      return_window_mass: bool = False):
-    """U[a][j] = sum_t A[a][t][j] for past columns j < n-w (Alg. 1 line 4).
+    """U[a][j] = sum_t A[a][t][j] for past columns j < n-w (Alg. 1 (past-only column sum U)).
 
     q_obs [H_q][w][d], k [n][H_k][d], float64; query head a reads kv head
-    a // group (contiguous groups, the Reshape([B,H_k,G,.]) of Alg. 1 line 6).
+    a // group (contiguous groups, the Reshape([B,H_k,G,.]) of Alg. 1 (SumGroups)).
     Returns U [H_q][n-w]; optionally also the mass that fell on the window's
     own columns, [H_q], so that U.sum + window mass = w per head."""
     Hq, w, d = q_obs.shape
@@ -104,7 +104,7 @@ def past_column_sums(q_obs: np.ndarray, k: np.ndarray, group: int,
 
 
 # --------------------------------------------------------------------------
-# Algorithm 1, line 5: 1-D pooling, kernel S, stride 1, pad floor(S/2)
+# Algorithm 1: 1-D pooling, kernel S, stride 1, pad floor(S/2)
 # --------------------------------------------------------------------------
 def pool1d(U: np.ndarray, S: int, mode: int = POOL_AVG) -> np.ndarray:
     """Pool every row of U [rows][T] along the token axis.
@@ -125,10 +125,10 @@ def pool1d(U: np.ndarray, S: int, mode: int = POOL_AVG) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# Algorithm 1, line 6 and the "scores" formula of Section 4.1
+# Algorithm 1: SumGroups, and the "scores" formula of Section 4.1
 # --------------------------------------------------------------------------
 def sum_groups(Vp: np.ndarray, group: int) -> np.ndarray:
-    """P[h] = sum_{g<G} Vp[h*G + g]  (Alg. 1 line 6)."""
+    """P[h] = sum_{g<G} Vp[h*G + g]  (Alg. 1 (SumGroups))."""
     Hq, T = Vp.shape
     return Vp.reshape(Hq // group, group, T).sum(axis=1)
 
@@ -139,14 +139,14 @@ def aggregate_scores(P: np.ndarray) -> np.ndarray:
 
 
 def score_layer(q_obs: np.ndarray, k: np.ndarray, group: int, S: int, mode: int = POOL_AVG):
-    """Alg. 1 lines 3-6 for one request.  Returns (P [H_k][T], agg [T])."""
+    """Alg. 1 from the window softmax to SumGroups for one request.  Returns (P [H_k][T], agg [T])."""
     U = past_column_sums(q_obs, k, group)
     P = sum_groups(pool1d(U, S, mode), group)
     return P, aggregate_scores(P)
 
 
 # --------------------------------------------------------------------------
-# Algorithm 1, line 9: RankDesc
+# Algorithm 1: RankDesc
 # --------------------------------------------------------------------------
 def rank_desc(scores: np.ndarray) -> np.ndarray:
     """rank[j] = 0-based position of token j when tokens are ordered by score
@@ -159,13 +159,13 @@ def rank_desc(scores: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# Algorithm 2, lines 5-9: union of per-layer top-k, variance of ranks
+# Algorithm 2: union of per-layer top-k (J, U), variance of ranks (RelNormVar)
 # --------------------------------------------------------------------------
 def rank_statistic(R: np.ndarray, k: int) -> Tuple[int, int, float]:
-    """R [rows][T] integer rank rows of the latest layers (Alg. 2 line 5).
+    """R [rows][T] integer rank rows of the latest layers (Alg. 2 (stacked rank rows R)).
 
-    J = the k smallest ranks of each row (line 7), U = Unique(Flatten(J))
-    (line 8) = {j : some row has R[r][j] < k}; var_top = mean over U of the
+    J = the k smallest ranks of each row (TopKIndices), U = Unique(Flatten(J))
+    = {j : some row has R[r][j] < k}; var_top = mean over U of the
     population variance over rows of R[:, j] (Sec. 4.1 "var_top").
     Returns (num, m, var_top) with num = sum_{j in U} (rows*sum r^2 - (sum r)^2)
     as an exact integer, m = |U|, var_top = num / (rows^2 * m)."""
@@ -196,18 +196,18 @@ class SelectionController:
 
     def step(self, layer_idx: int, agg: np.ndarray) -> dict:
         T = agg.shape[0]
-        self.cache.append((layer_idx, rank_desc(agg)))          # Alg. 1 line 9
+        self.cache.append((layer_idx, rank_desc(agg)))          # Alg. 1 (RankDesc)
         self.cache = self.cache[-self.l_obs:]
         out = {"layer": layer_idx, "evaluated": False, "selected": False}
-        if layer_idx < self.l_min or len(self.cache) < 2:        # Alg. 2 lines 1-3
+        if layer_idx < self.l_min or len(self.cache) < 2:        # Alg. 2 (early return)
             return out
-        R = np.stack([r for _, r in self.cache])                 # line 5
-        k = min(self.budget - self.window, T)                    # line 6
-        num, m, var_top = rank_statistic(R, k)                   # lines 7-9
+        R = np.stack([r for _, r in self.cache])                 # stacked rank rows R
+        k = min(self.budget - self.window, T)                    # k
+        num, m, var_top = rank_statistic(R, k)                   # J, U, RelNormVar
         if self.init_var is None:
             self.init_var = var_top
         rel = var_top / self.init_var if self.init_var != 0 else float("nan")
-        sel = bool(rel < self.tau)                               # line 10
+        sel = bool(rel < self.tau)                               # threshold test
         out.update(evaluated=True, rows=R.shape[0], num=num, m=m, var_top=var_top,
                    rel=rel, selected=sel)
         if sel and self.selected_layer < 0:
@@ -216,15 +216,15 @@ class SelectionController:
 
 
 # --------------------------------------------------------------------------
-# Algorithm 1, lines 7-8 and 10: per-head top-k, window append, gather
+# Algorithm 1: k, per-head TopK, window append, and the gather K[I], V[I]
 # --------------------------------------------------------------------------
 def kept_count(budget: int, n: int, window: int) -> int:
-    """k = min(KV_budget, N_q) - W  (Alg. 1 line 7)."""
+    """k = min(KV_budget, N_q) - W  (Alg. 1 (k))."""
     return min(budget, n) - window
 
 
 def select_topk(P_row: np.ndarray, k: int, n: int, window: int) -> np.ndarray:
-    """I = Concat(TopK(P, k), I_w) for one (request, kv head) (Alg. 1 line 8).
+    """I = Concat(TopK(P, k), I_w) for one (request, kv head) (Alg. 1 (TopK and window append)).
 
     The k past tokens with the largest score, ties to the lower index, listed
     in ascending index order, followed by the window indices n-w .. n-1."""
@@ -235,6 +235,21 @@ def select_topk(P_row: np.ndarray, k: int, n: int, window: int) -> np.ndarray:
 
 
 def compact_rows(x: np.ndarray, idx: np.ndarray, head: int) -> np.ndarray:
-    """K[I] (or V[I]) for one kv head: rows of x [n][H_k][d] at idx (Alg. 1 line 10).
+    """K[I] (or V[I]) for one kv head: rows of x [n][H_k][d] at idx (Alg. 1 (K[I], V[I])).
     Works on any dtype; used on the raw bf16 bit patterns."""
     return x[idx, head, :]
+
+
+# --------------------------------------------------------------------------
+# Algorithm 2: one-shot token selection at the selection layer
+# --------------------------------------------------------------------------
+def select_tokens(agg: np.ndarray, budget: int, n: int, window: int) -> np.ndarray:
+    """select_idx = Unique(J_last u I_w) (Alg. 2 (one-shot selection)): J_last are the k tokens with the
+    smallest rank of the current layer, i.e. the k best aggregate scores (ties to the lower
+    index), I_w the window tokens T .. T+W-1; Unique sorts.  k = min(budget - W, T)."""
+    T = agg.shape[0]
+    k = min(budget - window, T)
+    rank = rank_desc(agg)
+    J_last = np.nonzero(rank < k)[0]
+    I_w = np.arange(T, T + window)
+    return np.unique(np.concatenate([J_last, I_w])).astype(np.int64)

@@ -19,7 +19,7 @@ ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
-           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse")
+           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -64,6 +64,7 @@ def _load() -> C.CDLL:
     lib.asl_score_layer.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_score_layer_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_window_lse.argtypes = [vp, vp, sz, vp, vp]
+    lib.asl_compact_rows.argtypes = [vp, vp, vp, vp, i64, vp]
     lib.asl_rank_stat.argtypes = [vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.asl_select_topk.argtypes = [vp, vp, i32, vp, vp, sz, vp]
     lib.asl_compact_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -176,6 +177,11 @@ def asl_compact_kv(ctx, k, v, idx, k_out, v_out, stream=None) -> None:
                                _stream_handle(stream)), "asl_compact_kv")
 
 
+def asl_compact_rows(ctx, x, idx, out, row_bytes, stream=None) -> None:
+    _check(_lib.asl_compact_rows(ctx, _ptr(x), _ptr(idx), _ptr(out), int(row_bytes), _stream_handle(stream)),
+           "asl_compact_rows")
+
+
 def asl_device_status(ctx, stream=None):
     where = C.c_int32(0)
     st = _lib.asl_device_status(ctx, _stream_handle(stream), C.byref(where))
@@ -194,7 +200,7 @@ def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
     shared by every call on the device, so calls that could overlap on the GPU
     must be ordered; T is limited to ASL_RANK_STATIC_MAX_T."""
     _check(_lib.asl_rank_desc_static(_ptr(scores), int(T), _ptr(rank_out), _stream_handle(stream)),
-           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse")
+           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows")
 
 
 # ---- a small holder of one plan's device buffers -------------------------------------

@@ -217,6 +217,13 @@ asl_status asl_compact_kv(asl_ctx* c, const void* k, const void* v, const int32_
   return asl_launch_compact(c, k, v, idx, k_out, v_out, static_cast<cudaStream_t>(stream));
 }
 
+asl_status asl_compact_rows(asl_ctx* c, const void* x, const int32_t* idx, void* out, int64_t row_bytes, void* stream) {
+  if (!c || !c->planned || !x || !idx || !out) return ASL_ERR_INVALID;
+  if (row_bytes < 16 || row_bytes % 16 || row_bytes / 16 > 0x7fffffff) return ASL_ERR_INVALID;
+  if (!aligned16(x) || !aligned16(out)) return ASL_ERR_INVALID;
+  return asl_launch_compact_rows(c, x, idx, out, row_bytes, static_cast<cudaStream_t>(stream));
+}
+
 asl_status asl_device_status(asl_ctx* c, void* stream, int32_t* where) {
   if (!c) return ASL_ERR_INVALID;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

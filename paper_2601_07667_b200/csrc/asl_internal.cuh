@@ -84,5 +84,8 @@ asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st);
 
+asl_status asl_launch_compact_rows(asl_ctx* c, const void* x, const int32_t* idx, void* out, int64_t row_bytes,
+                                   cudaStream_t st);
+
 constexpr int ASL_SIMT_KEY_TILE = 128;   // keys per block in the SIMT scorer
 constexpr int ASL_RANK_TILE = 2048;      // keys per block in the radix sort

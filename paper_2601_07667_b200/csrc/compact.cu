@@ -1,4 +1,4 @@
-// K/V compaction (Algorithm 1 line 10): out[h][r][:] = x[tok_off + idx[h][r]][h][:].
+// K/V compaction (Algorithm 1 (K[I], V[I])): out[h][r][:] = x[tok_off + idx[h][r]][h][:].
 // 16 threads move one 256-byte row as 16-byte vectors; K and V in one launch.
 #include "asl_internal.cuh"
 
@@ -24,7 +24,31 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const uint16_t* __restr
   *reinterpret_cast<uint4*>(v_out + o) = vv;
 }
 
+// Row gather of one tensor with rows of `row_bytes` (a multiple of 16): out[kept_off_b + r] = x[tok_off_b + idx[r]].
+// A warp moves one row, 16 bytes per lane per trip.
+__global__ void __launch_bounds__(256) compact_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ idx,
+                                                           const AslReq* __restrict__ req, int vec_per_row,
+                                                           uint4* __restrict__ out) {
+  const int b = blockIdx.y;
+  const AslReq rq = req[b];
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= rq.kept) return;
+  const int64_t src = ((int64_t)rq.tok_off + idx[rq.kept_off + r]) * vec_per_row;
+  const int64_t dst = ((int64_t)rq.kept_off + r) * vec_per_row;
+  for (int c = lane; c < vec_per_row; c += 32) out[dst + c] = x[src + c];
+}
+
 }  // namespace
+
+asl_status asl_launch_compact_rows(asl_ctx* c, const void* x, const int32_t* idx, void* out, int64_t row_bytes,
+                                   cudaStream_t st) {
+  dim3 grid((c->max_kept + 7) / 8, c->p.batch);
+  compact_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(x), idx, c->d_req, (int)(row_bytes / 16),
+                                            static_cast<uint4*>(out));
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}
 
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st) {

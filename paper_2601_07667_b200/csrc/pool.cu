@@ -1,4 +1,4 @@
-// 1-D pooling, GQA group sum and all-head aggregate (Algorithm 1 lines 5-6 and
+// 1-D pooling, GQA group sum and all-head aggregate (Algorithm 1 (1-D pooling, SumGroups) and
 // the "scores" sum of Section 4.1).  One thread per past token walks the kv
 // heads, so the aggregate needs no atomics and is bit-reproducible.
 //   average pooling: input is group-summed column sums, `urows` rows per kv head

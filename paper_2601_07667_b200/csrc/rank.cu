@@ -1,4 +1,4 @@
-// Rank row and rank-variance statistic (Algorithm 1 line 9; Algorithm 2 lines 5-10;
+// Rank row and rank-variance statistic (Algorithm 1 (RankDesc); Algorithm 2 (stacked rank rows R, k, TopKIndices J, Unique U, RelNormVar, threshold test);
 // Section 4.1 "var_top" and "relative variance").
 //
 // RankDesc: stable least-significant-digit radix sort (8-bit digits) of

@@ -1,4 +1,4 @@
-// Observation-window scorer on the CUDA cores (Algorithm 1 lines 3-4).
+// Observation-window scorer on the CUDA cores (Algorithm 1 (window softmax A, past-only column sum U)).
 //
 // Two passes over K, both in the log2 domain x = (q.k) * log2(e)/sqrt(d):
 //   pass 1  thread = query row: online row max / row sum over one key tile,

@@ -1,4 +1,4 @@
-// Observation-window scorer on the 5th-generation tensor cores (Algorithm 1 lines 3-4).
+// Observation-window scorer on the 5th-generation tensor cores (Algorithm 1 (window softmax A, past-only column sum U)).
 //
 // One persistent kernel, one CTA per SM, does both softmax passes of every
 // (request, kv head, row chunk) "segment":

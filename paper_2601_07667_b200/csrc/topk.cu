@@ -1,4 +1,4 @@
-// Per-(request, head) top-k with the window appended (Algorithm 1 lines 7-8).
+// Per-(request, head) top-k with the window appended (Algorithm 1 (k, TopK and window append)).
 //
 // Radix select on an order-preserving 32-bit image of the fp32 score, 11+11+10
 // bits from the top: the exact k-th largest key is found; every token with a
@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(THREADS) topk_cluster_kernel(const float* __re
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int rounds = (T + CL * SLICE - 1) / (CL * SLICE);
 
-  // window indices (Algorithm 1 line 8)
+  // window indices (Algorithm 1 (TopK and window append))
   for (int t = r * THREADS + tid; t < rq.kept - k; t += CL * THREADS) out[k + t] = T + t;
   if (k == 0) return;                      // uniform over the cluster: nobody waits for anybody
 

@@ -226,3 +226,32 @@ def test_one_pass_scoring_with_supplied_lse(Hq, Hk, w, mode, n):
     assert np.abs(got.cpu().numpy()[0].astype(np.float64) - lse_ref).max() <= 2e-4     # log domain, absolute
     assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
     path.close()
+
+
+def test_one_shot_selection_and_hidden_state_gather():
+    """Alg. 2 (one-shot selection): top-k of the aggregate (one head) plus window, then a row gather of a
+    per-token tensor; ragged batch, rows of 200 bf16 values (400 bytes)."""
+    from paper_2601_07667_b200 import binding as B
+    wl = I.workload("C4", seqlens=(3000, 777, 4097), budgets=(300, 100, 5000), layers=1)
+    path = make_path(wl)
+    g = torch.Generator().manual_seed(5)
+    agg = torch.rand(path.sum_T, generator=g).mul(50).round().div(50)          # ties
+    hidden = torch.randn(wl.total_tokens, 200, generator=g).to(torch.bfloat16)
+    path.scores_agg.copy_(agg)
+    idx = torch.empty(path.sum_kept, dtype=torch.int32, device="cuda")
+    out = torch.empty(path.sum_kept, 200, dtype=torch.bfloat16, device="cuda")
+    hd = hidden.cuda()
+    B.asl_select_topk(path.ctx, path.scores_agg, 1, idx, path.workspace, path.ws_bytes)
+    B.asl_compact_rows(path.ctx, hd, idx, out, 400)
+    torch.cuda.synchronize()
+    idx_h, out_h = idx.cpu().numpy(), out.cpu()
+    cu = wl.cu_seqlens()
+    for b in range(wl.batch):
+        n, w = wl.seqlens[b], wl.window
+        ts, ko, kept = int(path.t_off[b]), int(path.kept_off[b]), wl.kept(b)
+        ref = O.select_tokens(agg[ts:ts + n - w].numpy().astype(np.float64), wl.budgets[b], n, w)
+        assert (idx_h[ko:ko + kept] == ref).all()
+        assert torch.equal(out_h[ko:ko + kept], hidden[int(cu[b]) + torch.from_numpy(ref)])
+    with pytest.raises(B.AslError):
+        B.asl_compact_rows(path.ctx, hd, idx, out, 100)                          # not a multiple of 16
+    path.close()

@@ -326,3 +326,16 @@ def test_window_lse_closed_form_and_brute_force():
             brute = math.log(math.fsum(math.exp(x) for x in logits))
             assert lse[a, t] == pytest.approx(brute, abs=1e-12)
             assert A[t, 3] == pytest.approx(math.exp(logits[3] - lse[a, t]), rel=1e-12)
+
+
+def test_select_tokens_is_the_union_of_best_ranks_and_window():
+    g = rng(33)
+    T, w, budget = 50, 6, 16
+    agg = g.integers(0, 8, size=T).astype(np.float64)          # many ties
+    sel = O.select_tokens(agg, budget, T + w, w)
+    k = budget - w
+    assert sel.shape[0] == k + w and (np.diff(sel) > 0).all()
+    assert (sel[k:] == np.arange(T, T + w)).all()
+    order = sorted(range(T), key=lambda j: (-agg[j], j))        # brute force: best k, ties to the lower index
+    assert sorted(order[:k]) == sel[:k].tolist()
+    assert (O.select_tokens(agg, 10 ** 6, T + w, w) == np.arange(T + w)).all()      # budget >= n keeps everything
