@@ -200,7 +200,7 @@ def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
     shared by every call on the device, so calls that could overlap on the GPU
     must be ordered; T is limited to ASL_RANK_STATIC_MAX_T."""
     _check(_lib.asl_rank_desc_static(_ptr(scores), int(T), _ptr(rank_out), _stream_handle(stream)),
-           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows")
+           "asl_rank_desc_static")
 
 
 # ---- a small holder of one plan's device buffers -------------------------------------
