@@ -408,8 +408,10 @@ def run_ours(args):
             "config": {"workload": wl.name, "seqlens": list(wl.seqlens), "window": wl.window,
                        "budgets": list(wl.budgets), "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv", "d": wl.head_dim,
                        "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"],
-                       "l2": f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
-                             f"{work['k_bytes'] / 1e6:.0f} MB per layer",
+                       "l2": (f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
+                              f"{work['k_bytes'] / 1e6:.0f} MB per layer") if work["k_bytes"] * n_sets > 126e6 else
+                             (f"small workload: {n_sets} layer sets of {work['k_bytes'] / 1e6:.1f} MB K stay in L2 "
+                              f"(launch-latency bound, a parity configuration)"),
                        "score_ctas": args.score_ctas, "tail_streams": args.tail_streams, "parallelism": f"replicas x{world}"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
