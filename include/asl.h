@@ -133,6 +133,18 @@ asl_status asl_score_layer(asl_ctx* ctx, const void* q_obs, const void* k, float
 asl_status asl_score_layer_lse(asl_ctx* ctx, const void* q_obs, const void* k, const float* lse, float* scores_kv,
                                float* scores_agg, void* workspace, size_t workspace_bytes, void* stream);
 
+/* asl_score_layer in two halves, for callers that pipeline layers: the first
+ * half is the scoring proper (the window softmax and the past-only column sums
+ * of Algorithm 1; lse null = two passes, else as asl_score_layer_lse) and leaves
+ * its un-pooled sums in slot 0 or 1 of the workspace; the second half is the
+ * pooling, SumGroups and the aggregate.  The second half of layer l may run on
+ * another stream while the first half of layer l+1 fills the other slot.
+ * asl_score_layer = both halves on slot 0. */
+asl_status asl_score_columns(asl_ctx* ctx, const void* q_obs, const void* k, const float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t slot, void* stream);
+asl_status asl_pool_scores(asl_ctx* ctx, void* workspace, size_t workspace_bytes, int32_t slot, float* scores_kv,
+                           float* scores_agg, void* stream);
+
 /* Denominators found by the latest asl_score_layer call on this workspace, in
  * the layout asl_score_layer_lse takes: lse_out device fp32 [B][H_q][W]. */
 asl_status asl_window_lse(asl_ctx* ctx, const void* workspace, size_t workspace_bytes, float* lse_out, void* stream);
@@ -152,7 +164,8 @@ asl_status asl_rank_stat(asl_ctx* ctx, const float* scores_agg, int32_t layer_id
  * past tokens with the largest score, ties to the lower index, written in
  * ascending index order and followed by the window indices T_b .. n_b-1.
  * scores device [n_heads][sum_T] fp32; idx_out device int32 [n_heads][sum_kept].
- * n_heads is H_k for the per-head cache, 1 for a selection on the aggregate. */
+ * n_heads is H_k for the per-head cache, 1 for a selection on the aggregate
+ * (1 <= n_heads <= H_k, else ASL_ERR_INVALID). */
 asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
                            void* workspace, size_t workspace_bytes, void* stream);
 
@@ -185,7 +198,7 @@ asl_status asl_compact_rows(asl_ctx* ctx, const void* x, const int32_t* idx, voi
  * Such a caller can use neither asl_create/asl_plan (both allocate small device
  * tables) nor a workspace it has nowhere to take from.  This call needs no
  * context and no workspace: its sort scratch is a fixed array compiled into
- * the library (about 4.2 MiB of device memory on every GPU that loads the
+ * the library (about 4.5 MiB of device memory on every GPU that loads the
  * library, held until the process exits).
  *
  *   scores    device fp32 [T]   one request's aggregate scores

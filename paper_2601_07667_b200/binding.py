@@ -19,7 +19,8 @@ ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
-           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows")
+           "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows",
+           "asl_score_columns", "asl_pool_scores")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -64,6 +65,8 @@ def _load() -> C.CDLL:
     lib.asl_score_layer.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_score_layer_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_window_lse.argtypes = [vp, vp, sz, vp, vp]
+    lib.asl_score_columns.argtypes = [vp, vp, vp, vp, vp, sz, i32, vp]
+    lib.asl_pool_scores.argtypes = [vp, vp, sz, i32, vp, vp, vp]
     lib.asl_compact_rows.argtypes = [vp, vp, vp, vp, i64, vp]
     lib.asl_rank_stat.argtypes = [vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.asl_select_topk.argtypes = [vp, vp, i32, vp, vp, sz, vp]
@@ -155,6 +158,16 @@ def asl_score_layer(ctx, q_obs, k, scores_kv, scores_agg, workspace, workspace_b
 def asl_score_layer_lse(ctx, q_obs, k, lse, scores_kv, scores_agg, workspace, workspace_bytes, stream=None) -> None:
     _check(_lib.asl_score_layer_lse(ctx, _ptr(q_obs), _ptr(k), _ptr(lse), _ptr(scores_kv), _ptr(scores_agg),
                                     _ptr(workspace), int(workspace_bytes), _stream_handle(stream)), "asl_score_layer_lse")
+
+
+def asl_score_columns(ctx, q_obs, k, lse, workspace, workspace_bytes, slot, stream=None) -> None:
+    _check(_lib.asl_score_columns(ctx, _ptr(q_obs), _ptr(k), _ptr(lse), _ptr(workspace), int(workspace_bytes), int(slot),
+                                  _stream_handle(stream)), "asl_score_columns")
+
+
+def asl_pool_scores(ctx, workspace, workspace_bytes, slot, scores_kv, scores_agg, stream=None) -> None:
+    _check(_lib.asl_pool_scores(ctx, _ptr(workspace), int(workspace_bytes), int(slot), _ptr(scores_kv), _ptr(scores_agg),
+                                _stream_handle(stream)), "asl_pool_scores")
 
 
 def asl_window_lse(ctx, workspace, workspace_bytes, lse_out, stream=None) -> None:
@@ -310,17 +323,18 @@ class LayerPath:
         if score_marks is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(main)
-        if lse is None:
-            asl_score_layer(ctx, q_obs, k, skv, agg, ws, wsb)
-        else:                                               # the caller holds the window rows' log-sum-exp: one pass
-            asl_score_layer_lse(ctx, q_obs, k, lse, skv, agg, ws, wsb)
+        asl_score_columns(ctx, q_obs, k, lse, ws, wsb, self._cur)      # lse: the window rows' log-sum-exp, or None
         if score_marks is not None:
             e1.record(main)
             score_marks.append((e0, e1))
         if overlap:
             self._fork.record(main)
             self.side.wait_event(self._fork)
-            self.side2.wait_event(self._fork)
+        asl_pool_scores(ctx, ws, wsb, self._cur, skv, agg, self.side if overlap else main)
+        if overlap and self.side2 is not self.side:
+            pooled = torch.cuda.Event()
+            pooled.record(self.side)
+            self.side2.wait_event(pooled)
         s1, s2 = (self.side, self.side2) if overlap else (main, main)
         asl_rank_stat(ctx, agg, layer_idx, rows, self.rank_ring, self.stat, ws, wsb, s1)
         asl_select_topk(ctx, skv, self.H_k, self.idx, ws, wsb, s2)

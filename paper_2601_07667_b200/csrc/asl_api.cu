@@ -143,13 +143,14 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   w.score_partials = off; off = asl_align256(off + partial_bytes);
   w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * c->rows_per_kv * sizeof(float));
   const size_t u_rows = (size_t)p->n_kv_heads * c->u_rows_per_kv;
-  w.score_u = off;        off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float));
+  for (int i = 0; i < 2; ++i) { w.score_u[i] = off; off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float)); }
   w.score_end = off;
   for (int i = 0; i < 2; ++i) { w.rank_keys[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
   for (int i = 0; i < 2; ++i) { w.rank_idx[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
   const size_t nblk = (max_T + ASL_RANK_TILE - 1) / ASL_RANK_TILE;
-  w.rank_hist = off;      off = asl_align256(off + (size_t)p->batch * 256 * nblk * sizeof(int32_t));
+  w.rank_hist = off;      off = asl_align256(off + (size_t)4 * p->batch * 256 * nblk * sizeof(int32_t));
   w.rank_end = off;
+  w.topk_scratch = off;   off = asl_align256(off + asl_topk_scratch_bytes((int64_t)p->batch * p->n_kv_heads, max_T));
   w.topk_end = off;
   w.total = off;
   *workspace_bytes = w.total;
@@ -165,27 +166,48 @@ asl_status asl_plan_sizes(const asl_ctx* c, int64_t* sum_tokens, int64_t* sum_T,
   return ASL_OK;
 }
 
-static asl_status score_layer_impl(asl_ctx* c, const void* q_obs, const void* k, const float* lse, float* scores_kv,
-                                   float* scores_agg, void* workspace, size_t workspace_bytes, void* stream) {
-  if (!c || !c->planned || !q_obs || !k || !scores_kv || !scores_agg) return ASL_ERR_INVALID;
+// scoring alone: un-pooled column sums into slot `slot` of the workspace
+static asl_status score_columns_impl(asl_ctx* c, const void* q_obs, const void* k, const float* lse, void* workspace,
+                                     size_t workspace_bytes, int slot, void* stream) {
+  if (!c || !c->planned || !q_obs || !k || slot < 0 || slot > 1) return ASL_ERR_INVALID;
   if (!aligned16(q_obs) || !aligned16(k)) return ASL_ERR_INVALID;
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
-  if (c->tc.enabled && !c->force_simt)
-    return asl_launch_score_tc(c, q_obs, k, lse, scores_kv, scores_agg, static_cast<char*>(workspace),
-                               static_cast<cudaStream_t>(stream));
-  return asl_launch_score_simt(c, q_obs, k, lse, scores_kv, scores_agg, static_cast<char*>(workspace),
-                               static_cast<cudaStream_t>(stream));
+  char* ws = static_cast<char*>(workspace);
+  float* u = reinterpret_cast<float*>(ws + c->ws.score_u[slot]);
+  if (c->tc.enabled && !c->force_simt) return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
+  return asl_launch_score_simt(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
+}
+
+static asl_status pool_scores_impl(asl_ctx* c, void* workspace, size_t workspace_bytes, int slot, float* scores_kv,
+                                   float* scores_agg, void* stream) {
+  if (!c || !c->planned || !scores_kv || !scores_agg || slot < 0 || slot > 1) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  const float* u = reinterpret_cast<const float*>(static_cast<char*>(workspace) + c->ws.score_u[slot]);
+  return asl_launch_pool(c, u, scores_kv, scores_agg, static_cast<cudaStream_t>(stream));
 }
 
 asl_status asl_score_layer(asl_ctx* c, const void* q_obs, const void* k, float* scores_kv, float* scores_agg,
                            void* workspace, size_t workspace_bytes, void* stream) {
-  return score_layer_impl(c, q_obs, k, nullptr, scores_kv, scores_agg, workspace, workspace_bytes, stream);
+  if (!scores_kv || !scores_agg) return ASL_ERR_INVALID;
+  const asl_status s = score_columns_impl(c, q_obs, k, nullptr, workspace, workspace_bytes, 0, stream);
+  return s != ASL_OK ? s : pool_scores_impl(c, workspace, workspace_bytes, 0, scores_kv, scores_agg, stream);
 }
 
 asl_status asl_score_layer_lse(asl_ctx* c, const void* q_obs, const void* k, const float* lse, float* scores_kv,
                                float* scores_agg, void* workspace, size_t workspace_bytes, void* stream) {
-  if (!lse) return ASL_ERR_INVALID;
-  return score_layer_impl(c, q_obs, k, lse, scores_kv, scores_agg, workspace, workspace_bytes, stream);
+  if (!lse || !scores_kv || !scores_agg) return ASL_ERR_INVALID;
+  const asl_status s = score_columns_impl(c, q_obs, k, lse, workspace, workspace_bytes, 0, stream);
+  return s != ASL_OK ? s : pool_scores_impl(c, workspace, workspace_bytes, 0, scores_kv, scores_agg, stream);
+}
+
+asl_status asl_score_columns(asl_ctx* c, const void* q_obs, const void* k, const float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t slot, void* stream) {
+  return score_columns_impl(c, q_obs, k, lse, workspace, workspace_bytes, slot, stream);
+}
+
+asl_status asl_pool_scores(asl_ctx* c, void* workspace, size_t workspace_bytes, int32_t slot, float* scores_kv,
+                           float* scores_agg, void* stream) {
+  return pool_scores_impl(c, workspace, workspace_bytes, slot, scores_kv, scores_agg, stream);
 }
 
 asl_status asl_window_lse(asl_ctx* c, const void* workspace, size_t workspace_bytes, float* lse_out, void* stream) {
@@ -206,8 +228,8 @@ asl_status asl_rank_stat(asl_ctx* c, const float* scores_agg, int32_t layer_idx,
 asl_status asl_select_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, void* workspace,
                            size_t workspace_bytes, void* stream) {
   if (!c || !c->planned || !scores || !idx_out || n_heads < 1) return ASL_ERR_INVALID;
-  if (!workspace || workspace_bytes < c->ws.total) return ASL_ERR_WORKSPACE;
-  return asl_launch_topk(c, scores, n_heads, idx_out, static_cast<cudaStream_t>(stream));
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  return asl_launch_topk(c, scores, n_heads, idx_out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
 }
 
 asl_status asl_compact_kv(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,

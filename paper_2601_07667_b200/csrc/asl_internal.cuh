@@ -24,13 +24,14 @@ struct AslReq {
 struct AslWorkspace {
   size_t score_partials;   // pass-1 partial row statistics
   size_t score_offsets;    // per-row log2 normalisers
-  size_t score_u;          // un-pooled column sums
+  size_t score_u[2];       // un-pooled column sums, two slots
   size_t score_end;
   size_t rank_keys[2];     // ping-pong sort keys
   size_t rank_idx[2];      // ping-pong sort payload
   size_t rank_hist;        // per-block digit histograms / offsets
   size_t rank_end;
-  size_t topk_end;         // (top-k keeps its state on chip)
+  size_t topk_scratch;     // per-segment digit histograms, pick state and per-tile counts
+  size_t topk_end;
   size_t total;
 };
 
@@ -68,19 +69,20 @@ struct asl_ctx {
 static inline size_t asl_align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 // ---- kernels' host launchers (one per translation unit) ----
-asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
-                                 float* scores_agg, char* ws, cudaStream_t st);
+asl_status asl_launch_score_simt(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
+                                 cudaStream_t st);
 asl_status asl_launch_window_lse(asl_ctx* c, const char* ws, float* lse_out, cudaStream_t st);
 bool asl_tc_plan(asl_ctx* c);
 void asl_tc_free(asl_ctx* c);
 size_t asl_tc_partial_bytes(const asl_ctx* c);
 asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st);
-asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
-                               float* scores_agg, char* ws, cudaStream_t st);
+asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
+                               cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);
-asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, cudaStream_t st);
+asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, char* ws, cudaStream_t st);
+size_t asl_topk_scratch_bytes(int64_t segments, int64_t max_T);
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st);
 

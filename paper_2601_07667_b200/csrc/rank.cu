@@ -1,7 +1,8 @@
 // Rank row and rank-variance statistic (Algorithm 1 (RankDesc); Algorithm 2 (stacked rank rows R, k, TopKIndices J, Unique U, RelNormVar, threshold test);
 // Section 4.1 "var_top" and "relative variance").
 //
-// RankDesc: stable least-significant-digit radix sort (8-bit digits) of
+// RankDesc: stable least-significant-digit radix sort (8-bit digits, one kernel
+// per digit after a first histogram) of
 // (key, token index) pairs per request, key = bit pattern that ascends as the
 // score descends; equal scores keep ascending index order, so the position of
 // a token in the sorted sequence is its 0-based rank with ties to the lower
@@ -60,13 +61,16 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ agg, const u
   }
 }
 
-// hist[b][blk][digit]: digit counts of one tile
-template <bool FIRST>
-__global__ void __launch_bounds__(SORT_THREADS) rank_hist(const float* __restrict__ agg, const uint32_t* __restrict__ keys,
-                                                          const AslReq* __restrict__ req, int shift, int nblk,
-                                                          int32_t* __restrict__ hist) {
+// hist[0][b][blk][digit]: digit counts of one tile of the scores, lowest digit.  The
+// tables of the three later passes are cleared here; each scatter pass counts the
+// next digit of what it writes into them.
+__global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __restrict__ agg, const AslReq* __restrict__ req,
+                                                                int nblk, int64_t table, int32_t* __restrict__ hist) {
   __shared__ int cnt[256];
   const int b = blockIdx.y, blk = blockIdx.x;
+  const int64_t row = ((int64_t)b * nblk + blk) * 256 + threadIdx.x;
+#pragma unroll
+  for (int t = 1; t < 4; ++t) hist[t * table + row] = 0;
   const AslReq rq = req[b];
   const int start = blk * TILE;
   if (start >= rq.T) return;
@@ -74,17 +78,17 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist(const float* __restric
   cnt[threadIdx.x] = 0;
   uint32_t key[ROUNDS];
   int32_t id[ROUNDS];
-  load_tile<FIRST>(agg, keys, nullptr, rq, start + wid * PER_WARP, lane, key, id);
+  load_tile<true>(agg, nullptr, nullptr, rq, start + wid * PER_WARP, lane, key, id);
   __syncthreads();
 #pragma unroll
   for (int r = 0; r < ROUNDS; ++r) {
     const bool valid = start + wid * PER_WARP + r * 32 + lane < rq.T;
-    const uint32_t d = (key[r] >> shift) & 255u;
+    const uint32_t d = key[r] & 255u;
     const uint32_t peers = same_digit(d, valid);
     if (valid && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&cnt[d], __popc(peers));
   }
   __syncthreads();
-  hist[((int64_t)b * nblk + blk) * 256 + threadIdx.x] = cnt[threadIdx.x];
+  hist[row] = cnt[threadIdx.x];
 }
 
 // in place: hist[b][blk][digit] -> first output position of (digit, blk), i.e. the
@@ -140,15 +144,22 @@ __global__ void __launch_bounds__(1024) rank_scan(int32_t* __restrict__ hist, co
   }
 }
 
-// stable scatter of one tile; on the last pass writes rank[token] = position
-template <bool FIRST>
+// Stable scatter of one tile; the last pass writes rank[token] = position.
+// SCAN: `counts` holds raw tile counts and the tile's first output positions are
+// summed here (thread = digit walks the tiles' rows; used while the request has few
+// tiles); otherwise `counts` was turned into positions by rank_scan.  A pass that is
+// not the last counts, per destination tile, the next digit of every pair it writes
+// (integer atomics: the table does not depend on the order of arrival).
+template <bool FIRST, bool SCAN>
 __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __restrict__ agg,
                                                              const uint32_t* __restrict__ keys_in,
                                                              const int32_t* __restrict__ idx_in,
                                                              uint32_t* __restrict__ keys_out, int32_t* __restrict__ idx_out,
-                                                             int32_t* __restrict__ rank_row, const int32_t* __restrict__ offs,
+                                                             int32_t* __restrict__ rank_row, const int32_t* __restrict__ counts,
+                                                             int32_t* __restrict__ next_counts,
                                                              const AslReq* __restrict__ req, int shift, int nblk) {
   __shared__ int cnt[WARPS][256];
+  __shared__ int warp_tot[WARPS];
   const int b = blockIdx.y, blk = blockIdx.x;
   const AslReq rq = req[b];
   const int start = blk * TILE;
@@ -159,7 +170,31 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
   uint32_t key[ROUNDS];
   int32_t id[ROUNDS];
   load_tile<FIRST>(agg, keys_in, idx_in, rq, wstart, lane, key, id);
-  const int tile_off = offs[((int64_t)b * nblk + blk) * 256 + threadIdx.x];
+  int tile_off;
+  if (SCAN) {
+    const int used = (rq.T + TILE - 1) / TILE;
+    const int32_t* col = counts + (int64_t)b * nblk * 256 + threadIdx.x;
+    int before = 0, total = 0;
+    for (int i0 = 0; i0 < used; i0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = (i0 + k < used) ? __ldcg(col + (int64_t)(i0 + k) * 256) : 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { total += v[k]; if (i0 + k < blk) before += v[k]; }
+    }
+    int incl = total;                       // exclusive scan of the digit totals over the 256 digits
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    tile_off = incl - total + before;
+    for (int w2 = 0; w2 < wid; ++w2) tile_off += warp_tot[w2];
+  } else {
+    tile_off = counts[((int64_t)b * nblk + blk) * 256 + threadIdx.x];
+  }
   for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&cnt[0][0])[i] = 0;
   __syncthreads();
   // per-warp digit counts; the peer masks are kept for the second walk
@@ -183,6 +218,8 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
     }
   }
   __syncthreads();
+  int32_t* next_b = next_counts ? next_counts + (int64_t)b * nblk * 256 : nullptr;
+  const bool top_next = shift == 16;        // the next digit is the sign/exponent byte: few distinct values
 #pragma unroll
   for (int r = 0; r < ROUNDS; ++r) {
     const bool valid = wstart + r * 32 + lane < rq.T;
@@ -196,28 +233,46 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
       if (rank_row) rank_row[rq.t_off + id[r]] = pos;
       else { keys_out[rq.t_off + pos] = key[r]; idx_out[rq.t_off + pos] = id[r]; }
     }
+    if (next_b) {
+      const uint32_t slot = valid ? (uint32_t)(pos / TILE) * 256u + ((key[r] >> (shift + 8)) & 255u) : 0xffffffffu;
+      if (top_next) {                       // one atomic per distinct counter of the warp
+        const uint32_t same = __match_any_sync(0xffffffffu, slot);
+        if (valid && (same & lt) == 0) atomicAdd(next_b + slot, __popc(same));
+      } else if (valid) {
+        atomicAdd(next_b + slot, 1);
+      }
+    }
   }
 }
 
-// the four passes of one rank row; scratch: two key and two index arrays, tile histograms
-void launch_sort(const float* agg, const AslReq* req, int batch, int max_T, uint32_t* const keys[2], int32_t* const idx[2],
-                 int32_t* hist, int32_t* rank_row, cudaStream_t st) {
+// the four passes of one rank row; scratch: two key and two index arrays, four tables of tile histograms
+constexpr int SCAN_IN_SCATTER_MAX_TILES = 128;
+
+int launch_sort(const float* agg, const AslReq* req, int batch, int max_T, uint32_t* const keys[2], int32_t* const idx[2],
+                int32_t* hist, int32_t* rank_row, cudaStream_t st) {
   const int nblk = (max_T + TILE - 1) / TILE;
   const dim3 grid(nblk, batch);
+  const int64_t table = (int64_t)batch * nblk * 256;
+  const bool fused_scan = nblk <= SCAN_IN_SCATTER_MAX_TILES;
+  int launches = 1;
+  rank_hist_first<<<grid, SORT_THREADS, 0, st>>>(agg, req, nblk, table, hist);
   for (int pass = 0; pass < 4; ++pass) {
     const int in = (pass + 1) & 1, out = in ^ 1;           // pass 0 reads the scores, writes buffer 0
     const int shift = pass * 8;
     int32_t* row = pass == 3 ? rank_row : nullptr;
+    int32_t* cur = hist + pass * table;
+    int32_t* nxt = pass == 3 ? nullptr : hist + (pass + 1) * table;
+    if (!fused_scan) { rank_scan<<<batch, 1024, 0, st>>>(cur, req, nblk); ++launches; }
+    ++launches;
     if (pass == 0) {
-      rank_hist<true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, req, shift, nblk, hist);
-      rank_scan<<<batch, 1024, 0, st>>>(hist, req, nblk);
-      rank_scatter<true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, hist, req, shift, nblk);
+      if (fused_scan) rank_scatter<true, true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, shift, nblk);
+      else rank_scatter<true, false><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, shift, nblk);
     } else {
-      rank_hist<false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], req, shift, nblk, hist);
-      rank_scan<<<batch, 1024, 0, st>>>(hist, req, nblk);
-      rank_scatter<false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, hist, req, shift, nblk);
+      if (fused_scan) rank_scatter<false, true><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, shift, nblk);
+      else rank_scatter<false, false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, shift, nblk);
     }
   }
+  return launches;
 }
 
 
@@ -307,8 +362,7 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
                      reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[1])};
   int32_t* hist = reinterpret_cast<int32_t*>(ws + c->ws.rank_hist);
   int32_t* row = ring + (int64_t)(layer_idx % p.l_obs) * c->sum_T;
-  launch_sort(agg, c->d_req, p.batch, c->max_T, keys, idx, hist, row, st);
-  c->launches += 12;
+  c->launches += launch_sort(agg, c->d_req, p.batch, c->max_T, keys, idx, hist, row, st);
   const int evaluate = (layer_idx >= p.l_min && n_rows >= 2) ? 1 : 0;
   if (evaluate) {
     StatArgs a{ring, c->d_req, c->d_acc, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows};
@@ -348,7 +402,7 @@ struct RankStaticScratch {
   AslReq req;                       // the one request the kernels index with blockIdx.y = 0
   uint32_t keys[2][STATIC_MAX_T];
   int32_t idx[2][STATIC_MAX_T];
-  int32_t hist[256 * STATIC_NBLK];
+  int32_t hist[4 * 256 * STATIC_NBLK];
 };
 
 static __device__ __align__(256) unsigned char g_rank_static[sizeof(RankStaticScratch)];

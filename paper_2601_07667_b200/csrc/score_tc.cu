@@ -340,7 +340,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   // ---- set-up: zero the Q buffers (rows past NC feed unused MMA rows), barriers, tensor memory ----
-  for (int i = threadIdx.x; i < 2 * Q_BUF_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
+  if (NC & 127)
+    for (int i = threadIdx.x; i < 2 * Q_BUF_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(BAR_FULL + s), 1); mbar_init(bar(BAR_EMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
@@ -851,8 +852,8 @@ asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st) {
   return ASL_OK;
 }
 
-asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* scores_kv,
-                               float* scores_agg, char* ws, cudaStream_t st) {
+asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
+                               cudaStream_t st) {
   const asl_params& p = c->p;
   AslTcPlan& tp = c->tc;
   const int W = p.window, G = p.n_q_heads / p.n_kv_heads, NC = tp.NC;
@@ -880,7 +881,6 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   a.req = c->d_req;
   a.partials = reinterpret_cast<float2*>(ws + c->ws.score_partials);
   a.offsets = reinterpret_cast<float*>(ws + c->ws.score_offsets);
-  float* u = reinterpret_cast<float*>(ws + c->ws.score_u);
   a.u = u;
   a.published = tp.d_sync;
   a.folded = tp.d_sync + tp.nseg;
@@ -899,5 +899,5 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   else                             score_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
-  return asl_launch_pool(c, u, scores_kv, scores_agg, st);
+  return ASL_OK;
 }

@@ -228,6 +228,38 @@ def test_one_pass_scoring_with_supplied_lse(Hq, Hk, w, mode, n):
     path.close()
 
 
+@pytest.mark.parametrize("Hq,Hk,w,mode,n", [(32, 8, 64, 0, 3000), (8, 2, 32, 1, 2000), (6, 2, 40, 0, 900)])
+def test_scoring_in_two_halves_matches_the_single_call_and_the_oracle(Hq, Hk, w, mode, n):
+    """asl_score_columns + asl_pool_scores on either workspace slot give the oracle's scores and,
+    bit for bit, what asl_score_layer gives; the two slots do not disturb each other."""
+    from paper_2601_07667_b200 import binding as B
+    from asl_check import assert_scores_close, oracle_layer
+    wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, pool_mode=mode, seqlens=(n,), budgets=(w + 50,),
+                    layers=2, l_min=1, l_obs=2)
+    xs = [I.layer_inputs(wl, l, seed=21) for l in range(2)]
+    path = make_path(wl)
+    qs, ks = [to_dev(x["q_obs"]) for x in xs], [to_dev(x["k"]) for x in xs]
+    whole = []
+    for l in range(2):
+        B.asl_score_layer(path.ctx, qs[l], ks[l], path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
+        whole.append((path.scores_kv.clone(), path.scores_agg.clone()))
+    # both first halves before either second half: slot 1 must survive the run that fills slot 0
+    B.asl_score_columns(path.ctx, qs[1], ks[1], None, path.workspace, path.ws_bytes, 1)
+    B.asl_score_columns(path.ctx, qs[0], ks[0], None, path.workspace, path.ws_bytes, 0)
+    for l in range(2):
+        kv, agg = torch.empty_like(path.scores_kv), torch.empty_like(path.scores_agg)
+        B.asl_pool_scores(path.ctx, path.workspace, path.ws_bytes, l, kv, agg)
+        torch.cuda.synchronize()
+        assert torch.equal(kv, whole[l][0]) and torch.equal(agg, whole[l][1])
+        P_ref, agg_ref = oracle_layer(wl, xs[l])
+        assert_scores_close(kv.cpu().numpy(), P_ref, "two-halves scores_kv")
+        assert_scores_close(agg.cpu().numpy(), agg_ref, "two-halves scores_agg")
+    with pytest.raises(B.AslError):
+        B.asl_score_columns(path.ctx, qs[0], ks[0], None, path.workspace, path.ws_bytes, 2)
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
 def test_one_shot_selection_and_hidden_state_gather():
     """Alg. 2 (one-shot selection): top-k of the aggregate (one head) plus window, then a row gather of a
     per-token tensor; ragged batch, rows of 200 bf16 values (400 bytes)."""
