@@ -438,9 +438,9 @@ def main():
     ap.add_argument("--layer-sets", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--tail-streams", type=int, default=1, choices=[1, 2],
+    ap.add_argument("--tail-streams", type=int, default=2, choices=[1, 2],
                     help="side streams for the rest of the layer: 2 = statistic and top-k/compaction side by side")
-    ap.add_argument("--score-ctas", type=int, default=-16,
+    ap.add_argument("--score-ctas", type=int, default=-24,
                     help="CTAs of the persistent scorer: 0 = one per SM, negative = that many fewer than SMs.  Fewer "
                          "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")
     ap.add_argument("--seqlens", type=str, default=None,

@@ -220,9 +220,9 @@ def asl_rank_desc_static(scores, T: int, rank_out, stream=None) -> None:
 class LayerPath:
     """Owns a context, its plan and the device buffers of one layer's pass
     (scores, indices, compacted cache, rank ring, statistic), all torch tensors.
-    ``run_layer`` issues the five steps: the scoring on the current stream, the
-    rest of the layer on a side stream (``tail_streams=2``: the rank statistic on
-    one, top-k and compaction on another) that is not waited for, so that it overlaps the scoring of the next layer (both
+    ``run_layer`` issues the five steps: the scoring proper on the current stream, the
+    rest of the layer (pooling first) on a side stream (``tail_streams=2``: pooling and the rank
+    statistic on one, top-k and compaction on another) that is not waited for, so that it overlaps the scoring of the next layer (both
     score buffers are double buffered for that; give the plan ``score_ctas``
     below the SM count to leave those kernels somewhere to run).  ``join`` makes
     the current stream wait for everything issued so far; ``read_stat`` joins by
