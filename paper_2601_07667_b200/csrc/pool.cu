@@ -16,14 +16,18 @@ namespace {
 constexpr int PT = 256;          // tokens per block
 constexpr int MAX_HALO = 16;     // pooling kernels up to 33 taps go through shared memory
 
-// One block pools PT consecutive past tokens of one request.  Row by row, the
-// un-pooled sums of the tile and its halo are staged in shared memory (partial
-// rows added on the way), pooled from there, and added up per kv head and over
-// all heads in a fixed order: no atomics, bit-reproducible.
+constexpr int HB = 8;            // staged rows per round: their loads are all in flight together
+
+// One block pools PT consecutive past tokens of one request.  A "unit" is what
+// gets pooled as one row: a kv head's group-summed sums (average pooling) or one
+// query head's sums (max pooling); it is stored as `nrows` consecutive partial
+// rows of u that are added on the way into shared memory.  HB units are staged
+// per round with their halo, pooled from there, and added up per kv head and
+// over all heads in a fixed order: no atomics, bit-reproducible.
 __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
                                                         int Hk, int G, int S, int mode, int urows, int parts, int64_t sum_T,
                                                         float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
-  __shared__ float tile[PT + 2 * MAX_HALO];
+  __shared__ float tile[HB][PT + 2 * MAX_HALO];
   const int b = blockIdx.y;
   const AslReq rq = req[b];
   const int j0 = blockIdx.x * PT;
@@ -33,42 +37,50 @@ __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict_
   const bool live = j < rq.T;
   const int lo = max(0, j - r), hi = min(rq.T - 1, j + r);
   const float inv = 1.0f / (float)S;
-  // stage sum over `nrows` consecutive rows starting at `row0` for tokens j0-r .. j0+PT-1+r (zero outside [0, T))
-  auto stage = [&](int row0, int nrows) {
+  const bool avg = mode == ASL_POOL_AVG;
+  const int units = avg ? Hk : Hk * G;
+  const int nrows = avg ? urows : parts;
+  const int per_head = avg ? 1 : G;
+  float agg = 0.f, p = 0.f;
+  for (int u0 = 0; u0 < units; u0 += HB) {
+    const int nb = min(HB, units - u0);
+    const int tot = nb * nrows;                       // rows u0*nrows .. u0*nrows + tot - 1 of u
     __syncthreads();
     for (int i = threadIdx.x; i < PT + 2 * r; i += PT) {
       const int t = j0 - r + i;
-      float v = 0.f;
-      if (t >= 0 && t < rq.T) {
-        const float* src = u + (int64_t)row0 * sum_T + rq.t_off + t;
-        for (int c = 0; c < nrows; ++c) v += src[(int64_t)c * sum_T];
+      const bool inside = t >= 0 && t < rq.T;
+      const float* src = u + (int64_t)u0 * nrows * sum_T + rq.t_off + t;
+#pragma unroll
+      for (int q = 0; q < HB; ++q) tile[q][i] = 0.f;
+      for (int e0 = 0; e0 < tot; e0 += 8) {
+        float x[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = (inside && e0 + k < tot) ? __ldcg(src + (int64_t)(e0 + k) * sum_T) : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (e0 + k < tot) tile[(e0 + k) / nrows][i] += x[k];
       }
-      tile[i] = v;
     }
     __syncthreads();
-  };
-  float agg = 0.f;
-  for (int h = 0; h < Hk; ++h) {
-    float p = 0.f;
-    if (mode == ASL_POOL_AVG) {
-      stage(h * urows, urows);
+    for (int q = 0; q < nb; ++q) {
       if (live) {
-        float s = 0.f;
-        for (int i = lo; i <= hi; ++i) s += tile[i - j0 + r];
-        p = s * inv;
-      }
-    } else {
-      for (int g = 0; g < G; ++g) {
-        stage((h * G + g) * parts, parts);
-        if (live) {
-          float mx = tile[lo - j0 + r];
-          for (int i = lo + 1; i <= hi; ++i) mx = fmaxf(mx, tile[i - j0 + r]);
+        if (avg) {
+          float s = 0.f;
+          for (int i = lo; i <= hi; ++i) s += tile[q][i - j0 + r];
+          p = s * inv;
+        } else {
+          float mx = tile[q][lo - j0 + r];
+          for (int i = lo + 1; i <= hi; ++i) mx = fmaxf(mx, tile[q][i - j0 + r]);
           p += mx;
         }
       }
+      const int unit = u0 + q;
+      if ((unit + 1) % per_head == 0) {
+        if (live) scores_kv[(int64_t)(unit / per_head) * sum_T + rq.t_off + j] = p;
+        agg += p;
+        p = 0.f;
+      }
     }
-    if (live) scores_kv[(int64_t)h * sum_T + rq.t_off + j] = p;
-    agg += p;
   }
   if (live) scores_agg[rq.t_off + j] = agg;
 }
