@@ -104,7 +104,8 @@ def test_max_pool_wide_gqa_small():
 def test_topk_exact_ties_lowest_index_wins():
     """Quantised scores: the k-th boundary falls inside long runs of exact ties."""
     from paper_2601_07667_b200 import binding as B
-    wl = I.workload("C1", seqlens=(9000 + 32, 2500 + 32), budgets=(1500, 2500 + 32))
+    # odd lengths: the second request's segment and every head's row start off a 16-byte boundary
+    wl = I.workload("C1", seqlens=(9001 + 32, 2503 + 32), budgets=(1500, 2503 + 32))
     path = make_path(wl)
     for levels in (3, 16, 200):
         s = I.quantised_scores(wl.n_kv_heads, path.sum_T, levels, seed=levels)
@@ -121,8 +122,8 @@ def test_topk_exact_ties_lowest_index_wins():
     path.close()
 
 
-def test_topk_long_segment_walked_in_rounds():
-    """A segment longer than one cluster's register cache (8 x 16384 scores)."""
+def test_topk_long_segment_of_many_tiles():
+    """A segment of 74 tiles: the k-th boundary and the runs of ties span tiles."""
     from paper_2601_07667_b200 import binding as B
     T, w = 300000, 32
     wl = I.workload("C1", seqlens=(T + w,), budgets=(5000,))
@@ -159,6 +160,23 @@ def test_rank_rows_with_ties_and_statistic_on_planted_rank_rows():
     B.asl_rank_stat(path.ctx, path.scores_agg, 2, 2, path.rank_ring, path.stat, path.workspace, path.ws_bytes)
     torch.cuda.synchronize()
     assert (path.rank_ring[0].cpu().numpy() == O.rank_desc(ties.cpu().numpy().astype(np.float64))).all()
+    path.close()
+
+
+def test_rank_row_of_a_long_segment():
+    """More tiles than the scatter kernel scans by itself: the separate scan kernel runs."""
+    from paper_2601_07667_b200 import binding as B
+    T, w = 300001, 32
+    wl = I.workload("C1", seqlens=(T + w,), budgets=(5000,), l_min=0, l_obs=2)
+    path = make_path(wl)
+    for layer, levels in enumerate((11, 1 << 20)):
+        s = I.quantised_scores(1, T, levels, seed=levels)[0]
+        s[::7] *= -1.0                                            # both signs
+        path.scores_agg.copy_(torch.from_numpy(s))
+        B.asl_rank_stat(path.ctx, path.scores_agg, layer, layer + 1, path.rank_ring, path.stat, path.workspace,
+                        path.ws_bytes)
+        torch.cuda.synchronize()
+        assert (path.rank_ring[layer % 2].cpu().numpy() == O.rank_desc(s.astype(np.float64))).all()
     path.close()
 
 
