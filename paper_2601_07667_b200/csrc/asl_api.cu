@@ -108,8 +108,8 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   free_plan(c);
   cudaError_t e = cudaMalloc(&c->d_req, sizeof(AslReq) * p->batch);
   if (e == cudaSuccess) e = cudaMemcpy(c->d_req, req.data(), sizeof(AslReq) * p->batch, cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMalloc(&c->d_acc, sizeof(unsigned long long) * 2 * p->batch);
-  if (e == cudaSuccess) e = cudaMemset(c->d_acc, 0, sizeof(unsigned long long) * 2 * p->batch);
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_acc, sizeof(unsigned long long) * (2 * p->batch + 1));
+  if (e == cudaSuccess) e = cudaMemset(c->d_acc, 0, sizeof(unsigned long long) * (2 * p->batch + 1));
   cudaSetDevice(prev);
   if (e != cudaSuccess) { free_plan(c); return ASL_ERR_CUDA; }
 

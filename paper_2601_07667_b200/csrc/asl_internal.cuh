@@ -47,7 +47,7 @@ struct asl_ctx {
   int64_t sum_tokens = 0, sum_T = 0, sum_kept = 0;
   int32_t max_n = 0, max_T = 0, max_kept = 0;
   AslReq* d_req = nullptr;            // device [B]
-  unsigned long long* d_acc = nullptr;  // device [B][2] integer accumulators of the statistic
+  unsigned long long* d_acc = nullptr;  // device [B][2] integer accumulators of the statistic + a block counter
   int32_t* d_err = nullptr;           // device error word of bounded waits
   // scorer plan
   int32_t rows_per_kv = 0;            // G*W

@@ -175,12 +175,12 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
     const int used = (rq.T + TILE - 1) / TILE;
     const int32_t* col = counts + (int64_t)b * nblk * 256 + threadIdx.x;
     int before = 0, total = 0;
-    for (int i0 = 0; i0 < used; i0 += 8) {
-      int v[8];
+    for (int i0 = 0; i0 < used; i0 += 32) {          // 32 loads in flight per thread
+      int v[32];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = (i0 + k < used) ? __ldcg(col + (int64_t)(i0 + k) * 256) : 0;
+      for (int k = 0; k < 32; ++k) v[k] = (i0 + k < used) ? __ldcg(col + (int64_t)(i0 + k) * 256) : 0;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) { total += v[k]; if (i0 + k < blk) before += v[k]; }
+      for (int k = 0; k < 32; ++k) { total += v[k]; if (i0 + k < blk) before += v[k]; }
     }
     int incl = total;                       // exclusive scan of the digit totals over the 256 digits
 #pragma unroll
@@ -279,10 +279,45 @@ int launch_sort(const float* agg, const AslReq* req, int batch, int max_T, uint3
 struct StatArgs {
   const int32_t* ring;
   const AslReq* req;
-  unsigned long long* acc;   // [B][2]: numerator, union size
+  unsigned long long* acc;   // [B][2]: numerator, union size; then one counter of finished blocks
+  asl_stat* stat;
   int64_t sum_T;
-  int32_t l_obs, first_layer, n_rows;
+  int32_t l_obs, first_layer, n_rows, batch, layer_idx;
+  double tau;
 };
+
+// Algorithm 2 (threshold test) for request b from the accumulated integers; clears them for the next layer
+__device__ void stat_finalize_one(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat, int b,
+                                  int layer_idx, int n_rows, int evaluate, double tau) {
+  asl_stat s = stat[b];
+  s.layer_idx = layer_idx;
+  s.k = req[b].k;
+  s.rows = n_rows;
+  s.evaluated = 0;
+  s.selected = 0;
+  s.num = 0;
+  s.m = 0;
+  if (evaluate) {
+    const unsigned long long num = __ldcg(acc + 2 * b), m = __ldcg(acc + 2 * b + 1);
+    acc[2 * b] = 0;
+    acc[2 * b + 1] = 0;
+    s.num = (int64_t)num;
+    s.m = (int32_t)m;
+    s.evaluated = 1;
+    s.var_top = (double)num / ((double)n_rows * (double)n_rows * (double)m);   // empty union (k = 0): NaN, never selects
+    if (!s.has_init) { s.init_var = s.var_top; s.has_init = 1; }
+    s.rel = s.var_top / s.init_var;
+    s.selected = (s.rel < tau) ? 1 : 0;
+  }
+  stat[b] = s;
+}
+
+// layers before L_min (or with a single rank row): only the bookkeeping fields change
+__global__ void rank_stat_skip(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat, int batch,
+                               int layer_idx, int n_rows) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < batch) stat_finalize_one(acc, req, stat, b, layer_idx, n_rows, 0, 0.0);
+}
 
 __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   __shared__ unsigned long long s_num[8];
@@ -315,40 +350,25 @@ __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   if (lane == 0) { s_num[wid] = num; s_m[wid] = m; }
   __syncthreads();
+  __shared__ bool last;
   if (threadIdx.x == 0) {
     for (int w2 = 1; w2 < 8; ++w2) { num += s_num[w2]; m += s_m[w2]; }
     if (m) {
       atomicAdd(&a.acc[2 * b], num);
       atomicAdd(&a.acc[2 * b + 1], (unsigned long long)m);
     }
+    // the block that finishes last sees every block's sums and closes the statistic
+    __threadfence();
+    const unsigned long long blocks = (unsigned long long)gridDim.x * gridDim.y;
+    last = atomicAdd(&a.acc[2 * a.batch], 1ull) + 1 == blocks;
   }
-}
-
-__global__ void rank_stat_finalize(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat,
-                                   int batch, int layer_idx, int n_rows, int evaluate, double tau) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= batch) return;
-  asl_stat s = stat[b];
-  s.layer_idx = layer_idx;
-  s.k = req[b].k;
-  s.rows = n_rows;
-  s.evaluated = 0;
-  s.selected = 0;
-  s.num = 0;
-  s.m = 0;
-  if (evaluate) {
-    const unsigned long long num = acc[2 * b], m = acc[2 * b + 1];
-    acc[2 * b] = 0;
-    acc[2 * b + 1] = 0;
-    s.num = (int64_t)num;
-    s.m = (int32_t)m;
-    s.evaluated = 1;
-    s.var_top = (double)num / ((double)n_rows * (double)n_rows * (double)m);   // empty union (k = 0): NaN, never selects
-    if (!s.has_init) { s.init_var = s.var_top; s.has_init = 1; }
-    s.rel = s.var_top / s.init_var;
-    s.selected = (s.rel < tau) ? 1 : 0;
+  __syncthreads();
+  if (last) {
+    __threadfence();
+    for (int bb = threadIdx.x; bb < a.batch; bb += blockDim.x)
+      stat_finalize_one(a.acc, a.req, a.stat, bb, a.layer_idx, a.n_rows, 1, a.tau);
+    if (threadIdx.x == 0) a.acc[2 * a.batch] = 0;
   }
-  stat[b] = s;
 }
 
 }  // namespace
@@ -365,12 +385,11 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
   c->launches += launch_sort(agg, c->d_req, p.batch, c->max_T, keys, idx, hist, row, st);
   const int evaluate = (layer_idx >= p.l_min && n_rows >= 2) ? 1 : 0;
   if (evaluate) {
-    StatArgs a{ring, c->d_req, c->d_acc, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows};
+    StatArgs a{ring, c->d_req, c->d_acc, stat, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows, p.batch, layer_idx, p.tau};
     rank_stat_accumulate<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(a);
-    c->launches += 1;
+  } else {
+    rank_stat_skip<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows);
   }
-  rank_stat_finalize<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, evaluate,
-                                                         p.tau);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;
