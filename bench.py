@@ -32,7 +32,7 @@ METRIC = "obs-window score+select+compact: context tokens/s/layer"
 UNIT = "tokens/s/layer"
 # dram__bytes_read.sum + dram__bytes_write.sum of one scorer launch, from the ncu capture summarised in
 # profiles/score_tc_fused_c3_128k_dram_traffic.txt (set to None when the scorer changes until re-captured)
-SCORER_TRAFFIC_BYTES = {"C3": 285.3e6}
+SCORER_TRAFFIC_BYTES = {"C3": 283.2e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -390,7 +390,7 @@ def run_ours(args):
         achieved = work["flops"] / (score_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": tf, "unit": "TFLOP/s", "frac": achieved / tf}
     default_shape = not args.seqlens and not args.budgets
-    roof.update({"traffic": SCORER_TRAFFIC_BYTES.get(wl.name) if default_shape else None, "kernel": "asl_score_layer (scorer passes + pooling)", "kernel_ms": score_ms,
+    roof.update({"traffic": SCORER_TRAFFIC_BYTES.get(wl.name) if default_shape else None, "kernel": "score_tc_kernel (asl_score_columns: both softmax passes, one persistent launch)", "kernel_ms": score_ms,
                  "peak_source": pk["source"], "step_roofline_us": max(t_hbm, t_mma) * 1e6,
                  "step_frac": max(t_hbm, t_mma) / (ms_step * 1e-3)})
 
