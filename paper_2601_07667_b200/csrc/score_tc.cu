@@ -668,10 +668,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               tc_ld32_issue(addr + (uint32_t)(blk * 32), cur);
               tc_ld_wait(cur);
               if (blk + 1 == nblk) release();
-              const float2* no = reinterpret_cast<const float2*>(no_base + blk * 32);
+              const float4* no = reinterpret_cast<const float4*>(no_base + blk * 32);   // two column pairs per load
               const float bs = exp_sum32(cur, scale2, [&](int pi) {
-                const float2 v = no[pi];
-                return pk(v.x, v.y);
+                const float4 v = no[pi >> 1];
+                return (pi & 1) ? pk(v.z, v.w) : pk(v.x, v.y);
               });
               if (PER_Q) {                                         // W is a multiple of 32: a block never straddles heads
                 const int slot = (blk * 32) / a.W;

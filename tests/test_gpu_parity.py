@@ -91,6 +91,36 @@ def test_scorer_shapes(Hq, Hk, w, mode, n):
     run_stack(wl, seed=5)
 
 
+def test_logits_far_above_the_first_keys_of_a_row():
+    """Keys whose logit exceeds the row's reference (the maximum over its first 32 keys) by more than
+    fp32's exponent range, so that the plain pass-1 sums overflow: in the last 32 keys of a tile (redone
+    from registers), in the middle of a tile (the tile is redone with running maxima), twice in a row."""
+    from paper_2601_07667_b200 import binding as B
+    from asl_check import assert_scores_close, oracle_layer
+    Hq, Hk, w, n = 32, 8, 64, 3000
+    wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, seqlens=(n,), budgets=(w + 100,), layers=1, l_min=1,
+                    l_obs=2)
+    g = np.random.default_rng(12)
+    q = np.ones((1, Hq, w, wl.head_dim), np.float32) * (1.0 + 0.25 * (np.arange(w) % 4))[None, None, :, None]
+    k = g.normal(0.0, 0.25, size=(n, Hk, wl.head_dim)).astype(np.float32)
+    # q.k / sqrt(d) = 11.3 a (.. 19.8 a for the largest rows): 100 .. 400 nats above the other keys
+    for pos, a in ((100, 9.0), (128 * 7 + 40, 13.25), (128 * 7 + 41, 20.0), (128 * 15 + 127, 11.0), (128 * 16, 12.0)):
+        k[pos] = a
+    x = {"q_obs": I.f32_to_bf16_bits(q), "k": I.f32_to_bf16_bits(k)}
+    path = make_path(wl)
+    B.asl_score_layer(path.ctx, to_dev(x["q_obs"]), to_dev(x["k"]), path.scores_kv, path.scores_agg, path.workspace,
+                      path.ws_bytes)
+    torch.cuda.synchronize()
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    P_ref, agg_ref = oracle_layer(wl, x)
+    kv = path.scores_kv.cpu().numpy()
+    assert np.isfinite(kv).all()
+    assert_scores_close(kv, P_ref, "scores_kv with overflowing logits")
+    assert_scores_close(path.scores_agg.cpu().numpy(), agg_ref, "scores_agg with overflowing logits")
+    assert P_ref[:, 128 * 7 + 41].min() > 1.0            # the largest key carries the rows' mass
+    path.close()
+
+
 def test_ragged_batch_small():
     wl = I.workload("C4", seqlens=(3000, 5001, 2177, 4096), budgets=(300, 500, 217, 409), layers=3)
     run_stack(wl, seed=1)
