@@ -280,6 +280,30 @@ class LayerPath:
         """Aggregate scores of the latest layer (device fp32 [sum_T])."""
         return self._agg[self._cur]
 
+    def _fresh_events(self) -> None:
+        torch = self.torch
+        self._agg_free = [None, None]
+        self._fork, self._join, self._join2 = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+
+    def capture(self, steps):
+        """Records ``run_layer`` for every ``(q_obs, k, v, layer_idx)`` (or ``(..., lse)``) of ``steps``,
+        followed by ``join``, into one CUDA graph and returns it (a ``torch.cuda.CUDAGraph``):
+        ``replay()`` then issues the whole sequence - the side streams included - as a single
+        launch, which removes the host's per-launch cost and shortens the gaps between the
+        dependent kernels of the statistic and the top-k.  The tensors must stay alive and in
+        place; run the same steps once without the graph first (module loading, lazy set-up)."""
+        torch = self.torch
+        torch.cuda.synchronize(self.dev)
+        self._fresh_events()            # nothing recorded outside the capture may be waited for inside it
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for step in steps:
+                q_obs, k, v, layer_idx = step[:4]
+                self.run_layer(q_obs, k, v, layer_idx, lse=step[4] if len(step) > 4 else None)
+            self.join()
+        self._fresh_events()            # and nothing recorded inside it afterwards
+        return graph
+
     def join(self) -> None:
         """The current stream waits for the statistic work issued so far."""
         cur = self.torch.cuda.current_stream()

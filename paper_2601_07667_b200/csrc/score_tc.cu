@@ -291,7 +291,9 @@ struct TcArgs {
   uint32_t* folded;        // [segment] rows whose offset is written, accumulated over launches
   int32_t* err;
   int64_t sum_T;
-  uint32_t epoch;          // launch number, from 1
+  uint32_t* epoch_word;    // two-pass launches completed so far (the counters accumulate over launches); then a ticket word
+  uint32_t epoch_limit;    // beyond it the last CTA clears the counters instead of letting them wrap
+  int32_t nseg;
   int32_t n_phases, total_items, NC, W, G, Hk, Hq, u_rows_per_kv, u_parts;
   float scale_log2;
 };
@@ -334,6 +336,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t bars = sbase + SM_BAR;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM_MISC + 4);
+  volatile uint32_t* s_epoch = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC + 8);
   float* s_negoff = reinterpret_cast<float*>(smem + SM_NEGOFF);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = a.NC;
@@ -350,6 +353,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     mbar_init(bar(BAR_DRAIN), 1);
     *s_abort = 0;
+    // This launch's number.  It is read on the device, not passed by the host, so that a launch
+    // replayed from a CUDA graph still counts: no CTA of this launch can see the increment below,
+    // which the last CTA to leave makes.
+    uint32_t done = 0;
+    if (!a.lse) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(done) : "l"(a.epoch_word) : "memory");
+    *s_epoch = done + 1u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -361,6 +370,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  const uint32_t epoch = *s_epoch;
 
   if (warp == 0) {
     // =============================== TMA producer ===============================
@@ -495,7 +505,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const TcPhase p = a.phases[ph];
       if (p.pass != 1) continue;
       if ((int)blockIdx.x + hw * grid >= NC) continue;             // no row of this segment is ours
-      if (!word_wait(a.published + p.seg, a.epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 2048)) break;
+      if (!word_wait(a.published + p.seg, epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 2048)) break;
       const int first = p.g0 % grid;
       for (int row = blockIdx.x + hw * grid; row < NC; row += 2 * grid) {
         const float2* src = a.partials + (int64_t)p.seg * entries * NC + row;
@@ -568,7 +578,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           first_tile = true;
         } else {
           // the segment's offsets: wait until every row has been folded, then stage -offset for this set
-          if (!dead && !a.lse) dead = !word_wait(a.folded + p.seg, a.epoch * (uint32_t)NC, s_abort, 33, lane, 256);
+          if (!dead && !a.lse) dead = !word_wait(a.folded + p.seg, epoch * (uint32_t)NC, s_abort, 33, lane, 256);
           bar_sync(2 + set, 256);                                 // the set is done with the previous offsets
           if (st < NC) {
             float off;
@@ -723,6 +733,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
   if (threadIdx.x == 0 && *s_abort) atomicCAS(a.err, 0, *s_abort);
+  if (threadIdx.x == 0 && !a.lse) {
+    // the last CTA to leave closes the launch: next launch number, or a fresh start before the counters wrap
+    __threadfence();
+    if (atomicAdd(a.epoch_word + 1, 1u) == gridDim.x - 1u) {
+      a.epoch_word[1] = 0;
+      if (epoch >= a.epoch_limit) {
+        for (int i = 0; i < 2 * a.nseg; ++i) a.published[i] = 0;      // published and folded are contiguous
+        a.epoch_word[0] = 0;
+      } else {
+        a.epoch_word[0] = epoch;
+      }
+      __threadfence();
+    }
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -811,7 +835,7 @@ bool asl_tc_plan(asl_ctx* c) {
   tp.n_phases2 = (int32_t)only2.size();
   tp.total_items2 = (int32_t)g2;
 
-  const size_t sync_bytes = 2 * (size_t)tp.nseg * sizeof(uint32_t);
+  const size_t sync_bytes = (2 * (size_t)tp.nseg + 2) * sizeof(uint32_t);   // counters, launch number, exit ticket
   cudaError_t e = cudaMalloc(&tp.d_phases, tp.phases.size() * sizeof(TcPhase));
   if (e == cudaSuccess) e = cudaMalloc(&tp.d_phases2, only2.size() * sizeof(TcPhase));
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases2, only2.data(), only2.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
@@ -819,7 +843,6 @@ bool asl_tc_plan(asl_ctx* c) {
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases, tp.phases.data(), tp.phases.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(tp.d_sync, 0, sync_bytes);
   if (e != cudaSuccess) { asl_tc_free(c); return false; }
-  tp.epoch = 0;
   cudaFuncSetAttribute(score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   cudaFuncSetAttribute(score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (cudaGetLastError() != cudaSuccess) { asl_tc_free(c); return false; }
@@ -847,8 +870,7 @@ void asl_tc_free(asl_ctx* c) {
 asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st) {
   AslTcPlan& tp = c->tc;
   if (!tp.d_sync) return ASL_OK;
-  ASL_CUDA(cudaMemsetAsync(tp.d_sync, 0, 2 * (size_t)tp.nseg * sizeof(uint32_t), st));
-  tp.epoch = 0;
+  ASL_CUDA(cudaMemsetAsync(tp.d_sync, 0, (2 * (size_t)tp.nseg + 2) * sizeof(uint32_t), st));
   return ASL_OK;
 }
 
@@ -871,10 +893,6 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
     const cuuint32_t box[3] = {64, 1, (cuuint32_t)KT};
     if (!make_map(&tm_k, k, 3, dims, strides, box)) return ASL_ERR_CUDA;
   }
-  if (tp.epoch >= 0xFFFFFFFFu / (uint32_t)(2 * tp.grid > MAX_NC ? 2 * tp.grid : MAX_NC) - 1u) {   // the counters would wrap
-    const asl_status rs = asl_tc_reset_sync(c, st);
-    if (rs != ASL_OK) return rs;
-  }
   TcArgs a{};
   a.phases = lse ? tp.d_phases2 : tp.d_phases;
   a.lse = lse;
@@ -886,7 +904,9 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   a.folded = tp.d_sync + tp.nseg;
   a.err = c->d_err;
   a.sum_T = c->sum_T;
-  a.epoch = lse ? tp.epoch : ++tp.epoch;          // the one-pass launch does not touch the counters
+  a.epoch_word = tp.d_sync + 2 * tp.nseg;         // the one-pass launch touches neither the counters nor this
+  a.epoch_limit = 0xFFFFFFFFu / (uint32_t)(2 * tp.grid > MAX_NC ? 2 * tp.grid : MAX_NC) - 2u;
+  a.nseg = tp.nseg;
   a.n_phases = lse ? tp.n_phases2 : (int32_t)tp.phases.size();
   a.total_items = lse ? tp.total_items2 : tp.total_items;
   a.NC = NC; a.W = W; a.G = G; a.Hk = p.n_kv_heads; a.Hq = p.n_q_heads;

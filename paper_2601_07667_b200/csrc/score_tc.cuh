@@ -19,11 +19,10 @@ struct AslTcPlan {
   int grid = 0;         // CTAs of the persistent kernel (one per SM)
   int group = 0;        // segments whose pass 1 runs before their pass 2
   int32_t total_items = 0;
-  uint32_t epoch = 0;   // launches so far; the device counters accumulate over launches
   std::vector<TcPhase> phases;   // both passes
   TcPhase* d_phases = nullptr;
   int32_t n_phases2 = 0;         // the pass-2 phases alone (scoring with a supplied log-sum-exp)
   int32_t total_items2 = 0;
   TcPhase* d_phases2 = nullptr;
-  uint32_t* d_sync = nullptr;   // [nseg] publish counters, [nseg] folded-row counters
+  uint32_t* d_sync = nullptr;   // [nseg] publish counters, [nseg] folded-row counters, launch number, exit ticket
 };

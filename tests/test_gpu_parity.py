@@ -249,6 +249,40 @@ def test_run_twice_is_bitwise_identical():
         assert torch.equal(a, b)
 
 
+def test_layers_replayed_from_a_cuda_graph_match_the_calls():
+    """LayerPath.capture: four layers (side streams included) recorded once and replayed three
+    times give, each time, bit for bit what the same calls give; the scorer numbers its launches
+    on the device, so a replay is not mistaken for the launch that was recorded."""
+    from paper_2601_07667_b200 import binding as B
+    wl = I.workload("C1", layers=4, l_min=1, l_obs=3)
+    xs = [I.layer_inputs(wl, l, seed=6) for l in range(4)]
+    dev = [(to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])) for x in xs]
+    path = make_path(wl)
+    def snapshot():
+        torch.cuda.synchronize()
+        return [t.clone() for t in (path.scores_kv, path.scores_agg, path.idx, path.k_out, path.v_out, path.rank_ring,
+                                    path.stat)]
+    for l in range(4):
+        path.run_layer(*dev[l], l)
+    path.join()
+    want = snapshot()
+    path.reset()
+    graph = path.capture([(*dev[l], l) for l in range(4)])
+    for _ in range(3):
+        path.reset()
+        graph.replay()
+        got = snapshot()
+        assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+        for a, b in zip(got, want):
+            assert torch.equal(a, b)
+    for l in range(4):                        # calls after a capture still work
+        path.run_layer(*dev[l], l)
+    path.join()
+    torch.cuda.synchronize()
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
 @pytest.mark.parametrize("Hq,Hk,w,mode,n", [(32, 8, 64, 0, 3000), (8, 2, 32, 1, 2000), (6, 2, 40, 0, 900)])
 def test_one_pass_scoring_with_supplied_lse(Hq, Hk, w, mode, n):
     """asl_score_layer_lse fed the oracle's log-sum-exp gives the oracle's scores; asl_window_lse
