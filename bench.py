@@ -294,11 +294,21 @@ def run_ours(args):
     step_args = lambda i: tuple(dev_sets[i % n_sets][k] for k in ("q_obs", "k", "v")) + (i,)
     graph = None
     launches0 = B.asl_launch_count(path.ctx)
+    issue = "call by call"
     if args.graph:
-        graph = path.capture([step_args(args.warmup + i) for i in range(args.steps)])
-        launches = B.asl_launch_count(path.ctx) - launches0          # kernels recorded = kernels per replay
-        graph.replay()                                               # untimed: uploads the graph
-        torch.cuda.synchronize()
+        try:
+            graph = path.capture([step_args(args.warmup + i) for i in range(args.steps)])
+            launches = B.asl_launch_count(path.ctx) - launches0      # kernels recorded = kernels per replay
+            graph.replay()                                           # untimed: uploads the graph
+            torch.cuda.synchronize()
+            issue = "one CUDA graph of the K steps"
+        except RuntimeError as e:                                    # capture refused: time the calls themselves
+            graph = None
+            args.graph = False
+            issue = "call by call (graph capture failed: %s)" % str(e).splitlines()[0][:80]
+            torch.cuda.synchronize()
+            path._fresh_events()
+            launches0 = B.asl_launch_count(path.ctx)
     t_start, t_end = ev(), ev()
     barrier()
     t_start.record(stream)
@@ -440,7 +450,7 @@ def run_ours(args):
                               f"{work['k_bytes'] / 1e6:.0f} MB per layer") if work["k_bytes"] * n_sets > 126e6 else
                              (f"small workload: {n_sets} layer sets of {work['k_bytes'] / 1e6:.1f} MB K stay in L2 "
                               f"(launch-latency bound, a parity configuration)"),
-                       "score_ctas": args.score_ctas, "tail_streams": args.tail_streams, "issue": "one CUDA graph of the K steps" if args.graph else "call by call", "parallelism": f"replicas x{world}"},
+                       "score_ctas": args.score_ctas, "tail_streams": args.tail_streams, "issue": issue, "parallelism": f"replicas x{world}"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},

@@ -169,6 +169,22 @@ asl_status asl_rank_stat(asl_ctx* ctx, const float* scores_agg, int32_t layer_id
 asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* Algorithm 2 as a state machine on the device, for callers that issue all layers ahead of time (one CUDA
+ * graph of the prompt's layers) and cannot branch on a layer's result on the host.
+ *   ASL_CONTROLLER_REPORT (default): every asl_rank_stat call sorts and evaluates its layer.
+ *   ASL_CONTROLLER_LATCH: once a request's record says `selected`, it is final: later asl_rank_stat calls
+ *     leave the request's record (layer_idx = the selection layer) and its rank rows as they are and their
+ *     blocks exit at once; the host reads the records once, after the last layer.
+ * asl_select_topk_gated is asl_select_topk for the requests whose record (`stat`, device [B], as written by
+ * the asl_rank_stat call of layer `layer_idx` ordered before it) selected at exactly that layer; the lists of
+ * all other requests are left untouched.  With n_heads = 1 on scores_agg, called after every layer's
+ * asl_rank_stat, it leaves in idx_out the one-shot selection of Algorithm 2 for every request that selected. */
+enum { ASL_CONTROLLER_REPORT = 0, ASL_CONTROLLER_LATCH = 1 };
+asl_status asl_set_controller(asl_ctx* ctx, int32_t mode);
+asl_status asl_select_topk_gated(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
+                                 const asl_stat* stat, int32_t layer_idx, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+
 /* Algorithm 1 (K[I], V[I]): k_out[h][r][:] = k[cu_seqlens[b] + idx[h][r]][h][:] and
  * the same for v, r running over request b's kept segment.
  * k_out, v_out: device bf16 dense [H_k][sum_kept][d]. */

@@ -20,7 +20,7 @@ ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
            "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows",
-           "asl_score_columns", "asl_pool_scores")
+           "asl_score_columns", "asl_pool_scores", "asl_set_controller", "asl_select_topk_gated")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -65,6 +65,8 @@ def _load() -> C.CDLL:
     lib.asl_score_layer.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_score_layer_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_window_lse.argtypes = [vp, vp, sz, vp, vp]
+    lib.asl_set_controller.argtypes = [vp, i32]
+    lib.asl_select_topk_gated.argtypes = [vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.asl_score_columns.argtypes = [vp, vp, vp, vp, vp, sz, i32, vp]
     lib.asl_pool_scores.argtypes = [vp, vp, sz, i32, vp, vp, vp]
     lib.asl_compact_rows.argtypes = [vp, vp, vp, vp, i64, vp]
@@ -158,6 +160,19 @@ def asl_score_layer(ctx, q_obs, k, scores_kv, scores_agg, workspace, workspace_b
 def asl_score_layer_lse(ctx, q_obs, k, lse, scores_kv, scores_agg, workspace, workspace_bytes, stream=None) -> None:
     _check(_lib.asl_score_layer_lse(ctx, _ptr(q_obs), _ptr(k), _ptr(lse), _ptr(scores_kv), _ptr(scores_agg),
                                     _ptr(workspace), int(workspace_bytes), _stream_handle(stream)), "asl_score_layer_lse")
+
+
+ASL_CONTROLLER_REPORT, ASL_CONTROLLER_LATCH = 0, 1
+
+
+def asl_set_controller(ctx, mode: int) -> None:
+    _check(_lib.asl_set_controller(ctx, int(mode)), "asl_set_controller")
+
+
+def asl_select_topk_gated(ctx, scores, n_heads, idx_out, stat, layer_idx, workspace, workspace_bytes, stream=None) -> None:
+    _check(_lib.asl_select_topk_gated(ctx, _ptr(scores), int(n_heads), _ptr(idx_out), _ptr(stat), int(layer_idx),
+                                      _ptr(workspace), int(workspace_bytes), _stream_handle(stream)),
+           "asl_select_topk_gated")
 
 
 def asl_score_columns(ctx, q_obs, k, lse, workspace, workspace_bytes, slot, stream=None) -> None:
@@ -296,7 +311,9 @@ class LayerPath:
         torch.cuda.synchronize(self.dev)
         self._fresh_events()            # nothing recorded outside the capture may be waited for inside it
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+        # thread_local: calls that other host threads make meanwhile (a process group's watchdog,
+        # a clock sampler) neither end up in the graph nor invalidate the capture
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
             for step in steps:
                 q_obs, k, v, layer_idx = step[:4]
                 self.run_layer(q_obs, k, v, layer_idx, lse=step[4] if len(step) > 4 else None)

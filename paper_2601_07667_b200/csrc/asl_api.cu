@@ -229,7 +229,22 @@ asl_status asl_select_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
                            size_t workspace_bytes, void* stream) {
   if (!c || !c->planned || !scores || !idx_out || n_heads < 1) return ASL_ERR_INVALID;
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
-  return asl_launch_topk(c, scores, n_heads, idx_out, static_cast<char*>(workspace), static_cast<cudaStream_t>(stream));
+  return asl_launch_topk(c, scores, n_heads, idx_out, nullptr, 0, static_cast<char*>(workspace),
+                         static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_select_topk_gated(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* stat,
+                                 int32_t layer_idx, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!c || !c->planned || !scores || !idx_out || !stat || n_heads < 1 || layer_idx < 0) return ASL_ERR_INVALID;
+  if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  return asl_launch_topk(c, scores, n_heads, idx_out, stat, layer_idx, static_cast<char*>(workspace),
+                         static_cast<cudaStream_t>(stream));
+}
+
+asl_status asl_set_controller(asl_ctx* c, int32_t mode) {
+  if (!c || (mode != ASL_CONTROLLER_REPORT && mode != ASL_CONTROLLER_LATCH)) return ASL_ERR_INVALID;
+  c->controller = mode;
+  return ASL_OK;
 }
 
 asl_status asl_compact_kv(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,

@@ -40,6 +40,7 @@ struct asl_ctx {
   int sm_count = 0;
   bool planned = false;
   bool force_simt = false;            // set from ASL_FORCE_SIMT=1 at create time (debugging aid)
+  int controller = 0;                 // ASL_CONTROLLER_*: asl_set_controller
   int score_group = 0;                // set from ASL_SCORE_GROUP at create time (0: default phase grouping)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
@@ -81,7 +82,8 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);
-asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, char* ws, cudaStream_t st);
+asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* gate,
+                           int32_t gate_layer, char* ws, cudaStream_t st);
 size_t asl_topk_scratch_bytes(int64_t segments, int64_t max_T);
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st);

@@ -65,12 +65,14 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ agg, const u
 // tables of the three later passes are cleared here; each scatter pass counts the
 // next digit of what it writes into them.
 __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __restrict__ agg, const AslReq* __restrict__ req,
-                                                                int nblk, int64_t table, int32_t* __restrict__ hist) {
+                                                                const asl_stat* __restrict__ latch, int nblk, int64_t table,
+                                                                int32_t* __restrict__ hist) {
   __shared__ int cnt[256];
   const int b = blockIdx.y, blk = blockIdx.x;
   const int64_t row = ((int64_t)b * nblk + blk) * 256 + threadIdx.x;
 #pragma unroll
   for (int t = 1; t < 4; ++t) hist[t * table + row] = 0;
+  if (latch && latch[b].selected) return;              // the request's selection is final: no more rank rows
   const AslReq rq = req[b];
   const int start = blk * TILE;
   if (start >= rq.T) return;
@@ -94,10 +96,12 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __r
 // in place: hist[b][blk][digit] -> first output position of (digit, blk), i.e. the
 // exclusive scan in (digit, blk) order.  1024 threads: thread (part, digit) walks a
 // quarter of the tiles with its loads batched, the parts are chained through shared memory.
-__global__ void __launch_bounds__(1024) rank_scan(int32_t* __restrict__ hist, const AslReq* __restrict__ req, int nblk) {
+__global__ void __launch_bounds__(1024) rank_scan(int32_t* __restrict__ hist, const AslReq* __restrict__ req,
+                                                  const asl_stat* __restrict__ latch, int nblk) {
   __shared__ int part_tot[4][256];
   __shared__ int warp_tot[8];
   const int b = blockIdx.x;
+  if (latch && latch[b].selected) return;
   const int used = (req[b].T + TILE - 1) / TILE;             // tiles of this request
   const int d = threadIdx.x & 255, part = threadIdx.x >> 8;
   const int per = (used + 3) / 4;
@@ -157,10 +161,12 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
                                                              uint32_t* __restrict__ keys_out, int32_t* __restrict__ idx_out,
                                                              int32_t* __restrict__ rank_row, const int32_t* __restrict__ counts,
                                                              int32_t* __restrict__ next_counts,
-                                                             const AslReq* __restrict__ req, int shift, int nblk) {
+                                                             const AslReq* __restrict__ req,
+                                                             const asl_stat* __restrict__ latch, int shift, int nblk) {
   __shared__ int cnt[WARPS][256];
   __shared__ int warp_tot[WARPS];
   const int b = blockIdx.y, blk = blockIdx.x;
+  if (latch && latch[b].selected) return;
   const AslReq rq = req[b];
   const int start = blk * TILE;
   if (start >= rq.T) return;
@@ -248,28 +254,28 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
 // the four passes of one rank row; scratch: two key and two index arrays, four tables of tile histograms
 constexpr int SCAN_IN_SCATTER_MAX_TILES = 128;
 
-int launch_sort(const float* agg, const AslReq* req, int batch, int max_T, uint32_t* const keys[2], int32_t* const idx[2],
-                int32_t* hist, int32_t* rank_row, cudaStream_t st) {
+int launch_sort(const float* agg, const AslReq* req, const asl_stat* latch, int batch, int max_T, uint32_t* const keys[2],
+                int32_t* const idx[2], int32_t* hist, int32_t* rank_row, cudaStream_t st) {
   const int nblk = (max_T + TILE - 1) / TILE;
   const dim3 grid(nblk, batch);
   const int64_t table = (int64_t)batch * nblk * 256;
   const bool fused_scan = nblk <= SCAN_IN_SCATTER_MAX_TILES;
   int launches = 1;
-  rank_hist_first<<<grid, SORT_THREADS, 0, st>>>(agg, req, nblk, table, hist);
+  rank_hist_first<<<grid, SORT_THREADS, 0, st>>>(agg, req, latch, nblk, table, hist);
   for (int pass = 0; pass < 4; ++pass) {
     const int in = (pass + 1) & 1, out = in ^ 1;           // pass 0 reads the scores, writes buffer 0
     const int shift = pass * 8;
     int32_t* row = pass == 3 ? rank_row : nullptr;
     int32_t* cur = hist + pass * table;
     int32_t* nxt = pass == 3 ? nullptr : hist + (pass + 1) * table;
-    if (!fused_scan) { rank_scan<<<batch, 1024, 0, st>>>(cur, req, nblk); ++launches; }
+    if (!fused_scan) { rank_scan<<<batch, 1024, 0, st>>>(cur, req, latch, nblk); ++launches; }
     ++launches;
     if (pass == 0) {
-      if (fused_scan) rank_scatter<true, true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, shift, nblk);
-      else rank_scatter<true, false><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, shift, nblk);
+      if (fused_scan) rank_scatter<true, true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      else rank_scatter<true, false><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
     } else {
-      if (fused_scan) rank_scatter<false, true><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, shift, nblk);
-      else rank_scatter<false, false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, shift, nblk);
+      if (fused_scan) rank_scatter<false, true><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      else rank_scatter<false, false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
     }
   }
   return launches;
@@ -282,14 +288,15 @@ struct StatArgs {
   unsigned long long* acc;   // [B][2]: numerator, union size; then one counter of finished blocks
   asl_stat* stat;
   int64_t sum_T;
-  int32_t l_obs, first_layer, n_rows, batch, layer_idx;
+  int32_t l_obs, first_layer, n_rows, batch, layer_idx, latch;
   double tau;
 };
 
 // Algorithm 2 (threshold test) for request b from the accumulated integers; clears them for the next layer
 __device__ void stat_finalize_one(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat, int b,
-                                  int layer_idx, int n_rows, int evaluate, double tau) {
+                                  int layer_idx, int n_rows, int evaluate, double tau, int latch) {
   asl_stat s = stat[b];
+  if (latch && s.selected) return;                     // final: the record keeps the selection layer
   s.layer_idx = layer_idx;
   s.k = req[b].k;
   s.rows = n_rows;
@@ -314,9 +321,9 @@ __device__ void stat_finalize_one(unsigned long long* acc, const AslReq* __restr
 
 // layers before L_min (or with a single rank row): only the bookkeeping fields change
 __global__ void rank_stat_skip(unsigned long long* acc, const AslReq* __restrict__ req, asl_stat* __restrict__ stat, int batch,
-                               int layer_idx, int n_rows) {
+                               int layer_idx, int n_rows, int latch) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < batch) stat_finalize_one(acc, req, stat, b, layer_idx, n_rows, 0, 0.0);
+  if (b < batch) stat_finalize_one(acc, req, stat, b, layer_idx, n_rows, 0, 0.0, latch);
 }
 
 __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
@@ -327,7 +334,7 @@ __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   unsigned long long num = 0;
   int m = 0;
-  if (j < rq.T) {
+  if (j < rq.T && !(a.latch && a.stat[b].selected)) {
     long long s1 = 0, s2 = 0;
     int mn = 0x7fffffff;
     for (int r = 0; r < a.n_rows; ++r) {
@@ -366,7 +373,7 @@ __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   if (last) {
     __threadfence();
     for (int bb = threadIdx.x; bb < a.batch; bb += blockDim.x)
-      stat_finalize_one(a.acc, a.req, a.stat, bb, a.layer_idx, a.n_rows, 1, a.tau);
+      stat_finalize_one(a.acc, a.req, a.stat, bb, a.layer_idx, a.n_rows, 1, a.tau, a.latch);
     if (threadIdx.x == 0) a.acc[2 * a.batch] = 0;
   }
 }
@@ -382,13 +389,15 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
                      reinterpret_cast<int32_t*>(ws + c->ws.rank_idx[1])};
   int32_t* hist = reinterpret_cast<int32_t*>(ws + c->ws.rank_hist);
   int32_t* row = ring + (int64_t)(layer_idx % p.l_obs) * c->sum_T;
-  c->launches += launch_sort(agg, c->d_req, p.batch, c->max_T, keys, idx, hist, row, st);
+  const asl_stat* latch = c->controller == ASL_CONTROLLER_LATCH ? stat : nullptr;
+  c->launches += launch_sort(agg, c->d_req, latch, p.batch, c->max_T, keys, idx, hist, row, st);
   const int evaluate = (layer_idx >= p.l_min && n_rows >= 2) ? 1 : 0;
   if (evaluate) {
-    StatArgs a{ring, c->d_req, c->d_acc, stat, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows, p.batch, layer_idx, p.tau};
+    StatArgs a{ring, c->d_req, c->d_acc, stat, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows, p.batch, layer_idx,
+               latch ? 1 : 0, p.tau};
     rank_stat_accumulate<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(a);
   } else {
-    rank_stat_skip<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows);
+    rank_stat_skip<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, latch ? 1 : 0);
   }
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
@@ -483,7 +492,7 @@ extern "C" asl_status asl_rank_desc_static(const float* scores, int32_t T, int32
   rank_static_begin<<<1, 1, 0, st>>>(s, T);
   uint32_t* const keys[2] = {s->keys[0], s->keys[1]};
   int32_t* const idx[2] = {s->idx[0], s->idx[1]};
-  launch_sort(scores, req, 1, T, keys, idx, s->hist, rank_out, st);
+  launch_sort(scores, req, nullptr, 1, T, keys, idx, s->hist, rank_out, st);
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;
 }

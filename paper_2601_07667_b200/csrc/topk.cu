@@ -40,6 +40,8 @@ struct TopkArgs {
   int32_t* idx_out;
   int64_t sum_T, sum_kept;
   int32_t n_heads, max_tiles;
+  const asl_stat* gate;  // null, or: only requests whose statistic selected at layer `gate_layer` are worked on
+  int32_t gate_layer;
 };
 
 struct Segment {
@@ -49,6 +51,7 @@ struct Segment {
   int32_t* counts;
   int32_t* out;
   int T, k, kept, tile;
+  bool open;             // false: the gate keeps this request's list as it is
 };
 
 __device__ __forceinline__ Segment segment_of(const TopkArgs& a) {
@@ -56,6 +59,7 @@ __device__ __forceinline__ Segment segment_of(const TopkArgs& a) {
   const AslReq rq = a.req[b];
   const int64_t seg = (int64_t)b * a.n_heads + h;
   Segment s;
+  s.open = !a.gate || (a.gate[b].selected && a.gate[b].layer_idx == a.gate_layer);
   s.row = a.scores + (int64_t)h * a.sum_T + rq.t_off;
   s.hist = a.scratch + seg * SEG_INTS;
   s.state = s.hist + 3 * BINS;
@@ -145,7 +149,7 @@ __device__ __forceinline__ void tile_histogram(const Segment& s, const uint32_t 
 template <int STAGE>
 __global__ void __launch_bounds__(THREADS) topk_digit_kernel(TopkArgs a) {
   const Segment s = segment_of(a);
-  if (s.k == 0 || s.tile * TILE >= s.T) return;
+  if (!s.open || s.k == 0 || s.tile * TILE >= s.T) return;
   uint32_t key[PER_THREAD];
   load_keys(s, key);
   if (STAGE == 0) {
@@ -169,7 +173,7 @@ __global__ void __launch_bounds__(THREADS) topk_digit_kernel(TopkArgs a) {
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(TopkArgs a) {
   __shared__ int w_gt[THREADS / 32], w_eq[THREADS / 32];
   const Segment s = segment_of(a);
-  if (s.k == 0 || s.tile * TILE >= s.T) return;
+  if (!s.open || s.k == 0 || s.tile * TILE >= s.T) return;
   uint32_t key[PER_THREAD];
   load_keys(s, key);
   const int bin1 = __ldcg(s.state + 0), bin2 = __ldcg(s.state + 2), rem2 = __ldcg(s.state + 3);
@@ -205,7 +209,7 @@ __global__ void __launch_bounds__(THREADS) topk_emit_kernel(TopkArgs a) {
   const Segment s = segment_of(a);
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int tiles = max(1, (s.T + TILE - 1) / TILE);
-  if (s.tile >= tiles) return;
+  if (!s.open || s.tile >= tiles) return;
   for (int t = s.tile * THREADS + tid; t < s.kept - s.k; t += tiles * THREADS) s.out[s.k + t] = s.T + t;   // the window
   if (s.k == 0) return;
   uint32_t key[PER_THREAD];
@@ -265,7 +269,8 @@ size_t asl_topk_scratch_bytes(int64_t segments, int64_t max_T) {
   return (size_t)(segments * SEG_INTS + segments * tiles * 2) * sizeof(int32_t);
 }
 
-asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, char* ws, cudaStream_t st) {
+asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* gate,
+                           int32_t gate_layer, char* ws, cudaStream_t st) {
   if (n_heads > c->p.n_kv_heads) return ASL_ERR_INVALID;      // the scratch is sized for H_k heads
   const int tiles = c->max_T > 0 ? (c->max_T + TILE - 1) / TILE : 1;
   const int64_t segments = (int64_t)c->p.batch * n_heads;
@@ -279,6 +284,8 @@ asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
   a.sum_kept = c->sum_kept;
   a.n_heads = n_heads;
   a.max_tiles = tiles;
+  a.gate = gate;
+  a.gate_layer = gate_layer;
   ASL_CUDA(cudaMemsetAsync(a.scratch, 0, (size_t)segments * SEG_INTS * sizeof(int32_t), st));
   const dim3 grid(tiles, n_heads, c->p.batch);
   topk_digit_kernel<0><<<grid, THREADS, 0, st>>>(a);

@@ -249,6 +249,81 @@ def test_run_twice_is_bitwise_identical():
         assert torch.equal(a, b)
 
 
+def test_device_side_controller_latches_the_selection_and_gates_the_one_shot_topk():
+    """ASL_CONTROLLER_LATCH: Algorithm 2's state machine runs on the device.  After the layer at
+    which a request's statistic selects, its record and rank rows stay as they are, and
+    asl_select_topk_gated writes the one-shot selection at exactly that layer.  Reference: the
+    oracle's controller and select_tokens fed the GPU's own aggregate scores layer by layer."""
+    import dataclasses
+    from paper_2601_07667_b200 import binding as B
+    # a per-token salience that grows with depth: the ranking settles, the relative variance falls
+    base = I.workload("C4", seqlens=(3000, 5001, 2177), budgets=(300, 500, 217), layers=7, l_min=1, l_obs=3,
+                      salience_start=0.0, salience_step=0.5)
+    xs = [I.layer_inputs(base, l, seed=11) for l in range(base.layers)]
+    dev = [(to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])) for x in xs]
+
+    def run(wl, latch):
+        path = make_path(wl)
+        if latch:
+            B.asl_set_controller(path.ctx, B.ASL_CONTROLLER_LATCH)
+        sel = torch.full((1, path.sum_kept), -1, dtype=torch.int32, device="cuda")
+        aggs, stats, rings = [], [], []
+        for l in range(wl.layers):
+            path.run_layer(*dev[l], l, overlap=False)
+            B.asl_select_topk_gated(path.ctx, path.scores_agg, 1, sel, path.stat, l, path.workspace, path.ws_bytes)
+            torch.cuda.synchronize()
+            aggs.append(path.scores_agg.cpu().numpy().astype(np.float64))
+            stats.append(path.read_stat().copy())
+            rings.append(path.rank_ring.cpu().numpy().copy())
+        assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+        out = (path, aggs, stats, rings, sel.cpu().numpy()[0])
+        return out
+
+    # without a threshold nothing selects: the relative variances of every layer, per request
+    never = dataclasses.replace(base, tau=0.0)
+    path0, aggs, stats0, _, sel0 = run(never, latch=False)
+    assert (sel0 == -1).all()
+    rel = np.array([[st[b]["rel"] for b in range(base.batch)] for st in stats0 if st[0]["evaluated"]])
+    tau = float(min(np.median(rel[1:-1]), 0.999))                 # some requests select somewhere in the middle ...
+    t_off, kept_off = path0.t_off, path0.kept_off
+    path0.close()
+
+    wl = dataclasses.replace(base, tau=tau)
+    ctl = [O.SelectionController(wl.budgets[b], wl.window, wl.l_min, wl.l_obs, wl.tau) for b in range(wl.batch)]
+    at_sel = {}
+    for l in range(wl.layers):
+        for b in range(wl.batch):
+            T = wl.seqlens[b] - wl.window
+            if ctl[b].selected_layer < 0:                        # one shot: the controller stops observing afterwards
+                rec = ctl[b].step(l, aggs[l][t_off[b]:t_off[b] + T])
+                if ctl[b].selected_layer == l:
+                    at_sel[b] = rec
+    sel_layers = [c.selected_layer for c in ctl]
+    assert any(1 < s < wl.layers - 1 for s in sel_layers) and len(set(sel_layers)) > 1, (sel_layers, tau, rel)   # ... not all alike
+
+    path, aggs1, stats, rings, sel = run(wl, latch=True)
+    for l in range(wl.layers):
+        assert np.array_equal(aggs1[l], aggs[l])                 # same inputs, same scores, bit for bit
+    final = stats[-1]
+    for b in range(wl.batch):
+        T, kept = wl.seqlens[b] - wl.window, wl.kept(b)
+        ts, ko = int(t_off[b]), int(kept_off[b])
+        L = sel_layers[b]
+        if L < 0:
+            assert final[b]["selected"] == 0 and (sel[ko:ko + kept] == -1).all()
+            continue
+        ref = at_sel[b]
+        assert final[b]["selected"] == 1 and final[b]["layer_idx"] == L
+        assert int(final[b]["num"]) == ref["num"] and int(final[b]["m"]) == ref["m"] and int(final[b]["rows"]) == ref["rows"]
+        assert abs(final[b]["rel"] - ref["rel"]) <= 1e-13 * abs(ref["rel"])
+        for l in range(L, wl.layers):                            # record and rank rows frozen from the selection layer on
+            assert stats[l][b] == stats[L][b]
+            assert np.array_equal(rings[l][:, ts:ts + T], rings[L][:, ts:ts + T])
+        want = O.select_tokens(aggs[L][ts:ts + T], wl.budgets[b], wl.seqlens[b], wl.window)
+        assert np.array_equal(sel[ko:ko + kept], want)
+    path.close()
+
+
 def test_layers_replayed_from_a_cuda_graph_match_the_calls():
     """LayerPath.capture: four layers (side streams included) recorded once and replayed three
     times give, each time, bit for bit what the same calls give; the scorer numbers its launches
