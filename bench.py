@@ -188,14 +188,18 @@ def time_oracle(wl, layer_sets, steps, warmup, heads):
 def make_workload(args):
     """The named workload, optionally with other context lengths (profiling-sized cases)."""
     base = I.workload(args.workload, seed=args.seed)
-    if not args.seqlens and not args.budgets:
+    if not args.seqlens and not args.budgets and not args.heads:
         return base
     seqlens = tuple(int(x) for x in args.seqlens.split(",")) if args.seqlens else base.seqlens
     if args.budgets:
         budgets = tuple(int(x) for x in args.budgets.split(","))
     else:                                          # keep the workload's first budget, one per request
         budgets = tuple(min(base.budgets[0], n) for n in seqlens)
-    return I.workload(args.workload, seed=args.seed, seqlens=seqlens, budgets=budgets)
+    heads = {}
+    if args.heads:
+        hq, hk = (int(x) for x in args.heads.split(","))
+        heads = {"n_q_heads": hq, "n_kv_heads": hk}
+    return I.workload(args.workload, seed=args.seed, seqlens=seqlens, budgets=budgets, **heads)
 
 
 def run_reference(args):
@@ -427,7 +431,7 @@ def run_ours(args):
     else:
         achieved = work["flops"] / (score_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": tf, "unit": "TFLOP/s", "frac": achieved / tf}
-    default_shape = not args.seqlens and not args.budgets
+    default_shape = not args.seqlens and not args.budgets and not args.heads
     roof.update({"traffic": SCORER_TRAFFIC_BYTES.get(wl.name) if default_shape else None, "kernel": "score_tc_kernel (asl_score_columns: both softmax passes, one persistent launch)", "kernel_ms": score_ms,
                  "peak_source": pk["source"], "step_roofline_us": max(t_hbm, t_mma) * 1e6,
                  "step_frac": max(t_hbm, t_mma) / (ms_step * 1e-3)})
@@ -486,6 +490,7 @@ def main():
     ap.add_argument("--seqlens", type=str, default=None,
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")
+    ap.add_argument("--heads", type=str, default=None, help="query,kv head counts replacing the workload's (e.g. 28,4)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -141,7 +141,8 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   size_t partial_bytes = (size_t)tiles * p->n_kv_heads * c->rows_per_kv * sizeof(float2);
   if (tc && asl_tc_partial_bytes(c) > partial_bytes) partial_bytes = asl_tc_partial_bytes(c);
   w.score_partials = off; off = asl_align256(off + partial_bytes);
-  w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * c->rows_per_kv * sizeof(float));
+  const size_t rows_padded = tc && c->tc.nchunk * c->tc.NC > c->rows_per_kv ? (size_t)c->tc.nchunk * c->tc.NC : (size_t)c->rows_per_kv;
+  w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * rows_padded * sizeof(float));
   const size_t u_rows = (size_t)p->n_kv_heads * c->u_rows_per_kv;
   for (int i = 0; i < 2; ++i) { w.score_u[i] = off; off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float)); }
   w.score_end = off;

@@ -170,9 +170,10 @@ __global__ void lse_to_offsets(const float* __restrict__ lse, float* __restrict_
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) offsets[i] = lse[i] * 1.4426950408889634f;
 }
-__global__ void offsets_to_lse(const float* __restrict__ offsets, float* __restrict__ lse, int n) {
+// `stride`: offsets per kv head (the tensor-core scorer pads a kv head's rows to whole chunks)
+__global__ void offsets_to_lse(const float* __restrict__ offsets, float* __restrict__ lse, int n, int R, int stride) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) lse[i] = __ldcg(offsets + i) * 0.6931471805599453f;
+  if (i < n) lse[i] = __ldcg(offsets + (int64_t)(i / R) * stride + i % R) * 0.6931471805599453f;
 }
 
 }  // namespace
@@ -181,7 +182,9 @@ __global__ void offsets_to_lse(const float* __restrict__ offsets, float* __restr
 // [b][h][g*W + t] and [b][h*G + g][t] are the same linear order: contiguous groups.
 asl_status asl_launch_window_lse(asl_ctx* c, const char* ws, float* lse_out, cudaStream_t st) {
   const int n = c->p.batch * c->p.n_kv_heads * c->rows_per_kv;
-  offsets_to_lse<<<(n + 255) / 256, 256, 0, st>>>(reinterpret_cast<const float*>(ws + c->ws.score_offsets), lse_out, n);
+  const int stride = (c->tc.enabled && !c->force_simt) ? c->tc.nchunk * c->tc.NC : c->rows_per_kv;
+  offsets_to_lse<<<(n + 255) / 256, 256, 0, st>>>(reinterpret_cast<const float*>(ws + c->ws.score_offsets), lse_out, n,
+                                                  c->rows_per_kv, stride);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

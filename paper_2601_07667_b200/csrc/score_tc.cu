@@ -581,8 +581,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!dead && !a.lse) dead = !word_wait(a.folded + p.seg, epoch * (uint32_t)NC, s_abort, 33, lane, 256);
           bar_sync(2 + set, 256);                                 // the set is done with the previous offsets
           if (st < NC) {
-            float off;
-            if (a.lse) {                                          // supplied: natural log -> log2 domain
+            float off = INFINITY;                                 // a padding row: 2^(x - inf) = 0
+            if (st >= p.rows) {
+            } else if (a.lse) {                                   // supplied: natural log -> log2 domain
               const int r = p.chunk * NC + st;                    // row within the kv head: query head r / W, window row r % W
               off = __ldg(a.lse + ((int64_t)p.b * a.Hq + p.h * a.G + r / a.W) * a.W + r % a.W) * 1.4426950408889634f;
             } else {
@@ -784,12 +785,27 @@ bool asl_tc_plan(asl_ctx* c) {
   tp = AslTcPlan();
   const int W = p.window, G = p.n_q_heads / p.n_kv_heads, R = G * W;
   if (p.head_dim != 128 || W % 32 || W > MAX_NC) return false;
+  // Chunk of NC query rows (whole heads, a multiple of 64 rows, at most 256).  Max pooling wants the
+  // chunks to tile the G*W rows exactly (its column sums are kept per query head).  Average pooling
+  // sums all rows of a kv head anyway, so the last chunk may be padded: its extra rows are given an
+  // infinite offset in pass 2 and add nothing.  Fewest chunks first, then least padding.
   int NC = 0;
-  for (int m = MAX_NC / W; m >= 1; --m)
-    if (R % (m * W) == 0) { NC = m * W; break; }
-  if (NC < 64 || NC % 64 || R % NC) return false;
+  if (p.pool_mode == ASL_POOL_MAX) {
+    for (int m = MAX_NC / W; m >= 1; --m)
+      if (R % (m * W) == 0) { NC = m * W; break; }
+    if (NC < 64 || NC % 64 || R % NC) return false;
+  } else {
+    int best_chunks = 0;
+    for (int m = 1; m * W <= MAX_NC; ++m) {
+      const int nc = m * W;
+      if (nc % 64) continue;
+      const int chunks = (R + nc - 1) / nc;
+      if (!NC || chunks < best_chunks) { NC = nc; best_chunks = chunks; }
+    }
+    if (!NC) return false;
+  }
   tp.NC = NC;
-  tp.nchunk = R / NC;
+  tp.nchunk = (R + NC - 1) / NC;
   tp.grid = (p.score_ctas > 0 && p.score_ctas < c->sm_count) ? p.score_ctas : c->sm_count;
 
   // segments in (request, head, chunk) order; phases in groups: pass 1 of `group` segments, then their pass 2
@@ -817,6 +833,7 @@ bool asl_tc_plan(asl_ctx* c) {
     ph.pass = pass; ph.seg = s; ph.b = segs[s].b; ph.h = segs[s].h; ph.chunk = segs[s].chunk;
     ph.ncontrib = segs[s].tiles1 < tp.grid ? segs[s].tiles1 : tp.grid;    // CTAs with a tile in pass 1
     ph.T = c->req[ph.b].T; ph.t_off = c->req[ph.b].t_off; ph.tok_off = c->req[ph.b].tok_off;
+    ph.rows = R - ph.chunk * NC < NC ? R - ph.chunk * NC : NC;
     g += ph.ntiles;
     tp.phases.push_back(ph);
   };

@@ -9,7 +9,8 @@ constexpr int ASL_TC_KEY_TILE = 128;
 // its tiles are the global work items g0 .. g0 + ntiles - 1
 // (T, t_off, tok_off: the request's past length, score offset and first token, copied here so that
 // one record is all a role needs when it enters the phase)
-struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, pad; };
+// rows: query rows of the chunk that exist (the last chunk of a kv head may be padded up to NC)
+struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, rows; };
 
 struct AslTcPlan {
   bool enabled = false;

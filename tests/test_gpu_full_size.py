@@ -55,3 +55,11 @@ def test_c4_ragged_batch_full():
 def test_c5_wide_gqa_max_pool_full():
     wl = I.workload("C5")
     sweep(wl, 0, range(0, 2))
+
+
+def test_half_million_token_context():
+    """524352 tokens in one request (8q/2kv so that the oracle still takes seconds): 4097 key tiles per
+    segment, 256 rank tiles (the separate scan kernel), 128 top-k tiles, 32-bit offsets near 2^30."""
+    wl = I.workload("C3", n_q_heads=8, n_kv_heads=2, seqlens=(524288 + 64,), budgets=(8192,), layers=2, l_min=1,
+                    l_obs=2)
+    sweep(wl, 3, range(0, 2))

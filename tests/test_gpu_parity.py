@@ -84,6 +84,7 @@ def test_edge_shapes(seqlens, budgets, w, S):
     (4, 2, 256, 1, 1500),     # window as large as a chunk
     (4, 4, 64, 0, 1111),      # no grouping: 64-row chunk
     (6, 2, 32, 0, 1000),      # 96-row chunk
+    (28, 4, 64, 0, 2500),     # seven query heads per kv head: 448 rows in seven 64-row chunks
 ])
 def test_scorer_shapes(Hq, Hk, w, mode, n):
     wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, pool_mode=mode, seqlens=(n,), budgets=(w + 100,),
@@ -358,7 +359,8 @@ def test_layers_replayed_from_a_cuda_graph_match_the_calls():
     path.close()
 
 
-@pytest.mark.parametrize("Hq,Hk,w,mode,n", [(32, 8, 64, 0, 3000), (8, 2, 32, 1, 2000), (6, 2, 40, 0, 900)])
+@pytest.mark.parametrize("Hq,Hk,w,mode,n", [(32, 8, 64, 0, 3000), (8, 2, 32, 1, 2000), (6, 2, 40, 0, 900),
+                                            (28, 4, 64, 0, 1500), (6, 2, 32, 0, 700)])     # the last two: padded chunks
 def test_one_pass_scoring_with_supplied_lse(Hq, Hk, w, mode, n):
     """asl_score_layer_lse fed the oracle's log-sum-exp gives the oracle's scores; asl_window_lse
     returns the denominators the two-pass call found (tensor-core shapes and the CUDA-core fallback)."""
