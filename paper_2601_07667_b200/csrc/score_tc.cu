@@ -505,7 +505,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const TcPhase p = a.phases[ph];
       if (p.pass != 1) continue;
       if ((int)blockIdx.x + hw * grid >= NC) continue;             // no row of this segment is ours
-      if (!word_wait(a.published + p.seg, epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 2048)) break;
+      if (!word_wait(a.published + p.seg, epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 256)) break;
       const int first = p.g0 % grid;
       for (int row = blockIdx.x + hw * grid; row < NC; row += 2 * grid) {
         const float2* src = a.partials + (int64_t)p.seg * entries * NC + row;
