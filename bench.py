@@ -32,7 +32,7 @@ METRIC = "obs-window score+select+compact: context tokens/s/layer"
 UNIT = "tokens/s/layer"
 # dram__bytes_read.sum + dram__bytes_write.sum of one scorer launch, from the ncu capture summarised in
 # profiles/score_tc_fused_c3_128k_dram_traffic.txt (set to None when the scorer changes until re-captured)
-SCORER_TRAFFIC_BYTES = {"C3": 286.2e6}
+SCORER_TRAFFIC_BYTES = {"C3": 279.4e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

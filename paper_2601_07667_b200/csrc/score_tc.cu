@@ -131,10 +131,23 @@ __device__ __forceinline__ bool word_wait(const uint32_t* p, uint32_t want, vola
   return __shfl_sync(0xffffffffu, gave_up, 0) == 0;
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+// L2 eviction policies for the K stream: pass 1 asks L2 to keep what pass 2 will read again, pass 2
+// (and a launch that has only pass 2) marks what it reads as the first to go.
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-      "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;" ::"r"(dst),
+      "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
@@ -377,6 +390,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // Local phase l (the l-th phase in which this CTA has a tile) uses Q buffer l%2.
     if (lane == 0) {
       ItemWalk w(a);
+      const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
       int item = 0, lp = -1, cur_ph = -1;
       int q_issued = -1;                       // highest local phase whose Q chunk has been requested
       int loaded_seg[2] = {-1, -1};
@@ -430,8 +444,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_expect_tx(bar(BAR_FULL + s), STAGE_BYTES);
         const uint32_t dst = sbase + SM_K + s * STAGE_BYTES;
         const int tok = tok_off + (w.g - p.g0) * KT;
-        tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok);
-        tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok);
+        const uint64_t pol = p.pass == 1 ? pol_keep : pol_stream;
+        tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok, pol);
+        tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok, pol);
       }
       if (!ok) {
         // let the copies already issued land before the CTA's shared memory is released
