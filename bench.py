@@ -33,6 +33,9 @@ UNIT = "tokens/s/layer"
 # dram__bytes_read.sum + dram__bytes_write.sum of one scorer launch, from the ncu capture summarised in
 # profiles/score_tc_fused_c3_128k_dram_traffic.txt (set to None when the scorer changes until re-captured)
 SCORER_TRAFFIC_BYTES = {"C3": 279.4e6}
+# default launch configuration of the timed steps (the GPU parity tests build their paths from the same two values)
+DEFAULT_SCORE_CTAS = -16       # persistent scorer: this many CTAs fewer than SMs (0 = one per SM)
+DEFAULT_TAIL_STREAMS = 2       # side streams for the rest of the layer
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -116,6 +119,12 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(mhz), "reasons": sorted(reasons)}
 
 
+def default_launch(sm_count: int) -> dict:
+    """LayerPath keywords of the launch configuration this benchmark times by default."""
+    ctas = DEFAULT_SCORE_CTAS if DEFAULT_SCORE_CTAS > 0 else max(1, sm_count + DEFAULT_SCORE_CTAS)
+    return {"score_ctas": ctas, "tail_streams": DEFAULT_TAIL_STREAMS}
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -142,6 +151,46 @@ def max_over_ranks(ms: float, world: int, device="cuda") -> float:
 def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
     """Whole-job throughput: every rank's tokens over the slowest rank's step time."""
     return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
+def spawn_replicas(n: int, argv) -> int:
+    """Starts ``n`` ranks of this script on this node (rank r on GPU r), one process each, with the
+    rendezvous variables a launcher would set, and waits for them.  Returns the worst exit code.
+    Rank 0's JSON line goes to this process's stdout; the other ranks print nothing."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env))
+    worst = 0
+    for p in procs:
+        rc = p.wait()
+        worst = rc if rc != 0 and worst == 0 else worst
+    return worst
+
+
+def run_dry(args):
+    """Rendezvous only (no kernel runs, no GPU needed): every rank joins the process group (NCCL on a
+    CUDA box, gloo otherwise), the per-rank times 1+rank ms are MAX-reduced as the timed region's
+    would be, and rank 0 prints the distributed fields of the JSON line."""
+    import torch
+    import torch.distributed as dist
+    rank, world, local = dist_env()
+    cuda = torch.cuda.is_available()
+    if cuda:
+        torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl" if cuda else "gloo")
+    ms = max_over_ranks(1.0 + rank, world, device="cuda" if cuda else "cpu")
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "ms_per_step": ms, "seed_of_last_rank": rank_seed(args.seed, world - 1),
+                          "value": aggregate_tokens_per_s(1000, world, ms), "scaling": "weak"}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
 
 
 # --------------------------------------------------------------------------------------
@@ -395,10 +444,10 @@ def run_ours(args):
         k_d.view(torch.int16).copy_(hp["k"], non_blocking=True)
         v_d.view(torch.int16).copy_(hp["v"], non_blocking=True)
         path.run_layer(q_d, k_d, v_d, i)
+        path.join()                     # top-k, compaction and the statistic run on side streams
         idx_h.copy_(path.idx, non_blocking=True)
         ko_h.copy_(path.k_out, non_blocking=True)
         vo_h.copy_(path.v_out, non_blocking=True)
-        path.join()
         st_h.copy_(path.stat, non_blocking=True)
 
     path.reset()
@@ -411,6 +460,10 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / e2e_steps
+    # the leg checks what it timed: the host copies are the device results of the last step
+    if not (torch.equal(idx_h, path.idx.cpu()) and torch.equal(ko_h.view(torch.int16), path.k_out.cpu().view(torch.int16))
+            and torch.equal(st_h, path.stat.cpu())):
+        raise SystemExit("end-to-end leg: host copies differ from the device results")
     h2d = sum(host_pinned[0][k].numel() * 2 for k in ("q_obs", "k", "v"))
     d2h = idx_h.numel() * 4 + ko_h.numel() * 2 + vo_h.numel() * 2 + st_h.numel()
 
@@ -482,20 +535,31 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="issue the timed steps call by call instead of replaying one CUDA graph of them")
-    ap.add_argument("--tail-streams", type=int, default=2, choices=[1, 2],
+    ap.add_argument("--tail-streams", type=int, default=DEFAULT_TAIL_STREAMS, choices=[1, 2],
                     help="side streams for the rest of the layer: 2 = statistic and top-k/compaction side by side")
-    ap.add_argument("--score-ctas", type=int, default=-16,
+    ap.add_argument("--score-ctas", type=int, default=DEFAULT_SCORE_CTAS,
                     help="CTAs of the persistent scorer: 0 = one per SM, negative = that many fewer than SMs.  Fewer "
                          "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")
     ap.add_argument("--seqlens", type=str, default=None,
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")
     ap.add_argument("--heads", type=str, default=None, help="query,kv head counts replacing the workload's (e.g. 28,4)")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="ranks only rendezvous and reduce a fixed time (checks the multi-rank launch; runs no kernel)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+        return
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1:
+        # started without a launcher: this process becomes the launcher of the N replicas
+        raise SystemExit(spawn_replicas(args.gpus, sys.argv[1:]))
+    if world_env is not None and int(world_env) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started WORLD_SIZE={world_env} ranks")
+    if args.dry_run:
+        run_dry(args)
     else:
         run_ours(args)
 

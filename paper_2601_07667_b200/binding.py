@@ -11,7 +11,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("ASL_B200_LIB") or os.path.join(_HERE, "libasl_b200.so")
+LIB_PATH = os.path.join(_HERE, "libasl_b200.so")
 
 ASL_POOL_AVG, ASL_POOL_MAX = 0, 1
 ASL_OK, ASL_ERR_INVALID, ASL_ERR_UNSUPPORTED, ASL_ERR_WORKSPACE = 0, -1, -2, -3

@@ -1,4 +1,4 @@
-"""Builds libasl_b200.so (sm_100a) and the oracle's C parts, in-tree.
+"""Builds libasl_b200.so (sm_100a), in-tree.
 
     python -m paper_2601_07667_b200.build [--force] [--verbose]
 """

@@ -33,10 +33,6 @@ asl_status asl_create(asl_ctx** out, int device) {
   asl_ctx* c = new (std::nothrow) asl_ctx();
   if (!c) return ASL_ERR_CUDA;
   c->device = device;
-  const char* fs = getenv("ASL_FORCE_SIMT");
-  c->force_simt = fs && fs[0] == '1';
-  const char* sg = getenv("ASL_SCORE_GROUP");
-  c->score_group = sg ? atoi(sg) : 0;
   c->sm_count = prop.multiProcessorCount;
   int prev = 0;
   cudaGetDevice(&prev);
@@ -128,7 +124,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
 
   cudaGetDevice(&prev);
   cudaSetDevice(c->device);
-  const bool tc = asl_tc_plan(c) && !c->force_simt;
+  const bool tc = asl_tc_plan(c);
   cudaSetDevice(prev);
   const int G = p->n_q_heads / p->n_kv_heads;
   // the tensor-core scorer writes two partial column sums per chunk (one per half of the chunk's rows);
@@ -175,7 +171,7 @@ static asl_status score_columns_impl(asl_ctx* c, const void* q_obs, const void* 
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
   float* u = reinterpret_cast<float*>(ws + c->ws.score_u[slot]);
-  if (c->tc.enabled && !c->force_simt) return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
+  if (c->tc.enabled) return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
   return asl_launch_score_simt(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
 }
 

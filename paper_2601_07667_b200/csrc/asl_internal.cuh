@@ -39,9 +39,7 @@ struct asl_ctx {
   int device = 0;
   int sm_count = 0;
   bool planned = false;
-  bool force_simt = false;            // set from ASL_FORCE_SIMT=1 at create time (debugging aid)
   int controller = 0;                 // ASL_CONTROLLER_*: asl_set_controller
-  int score_group = 0;                // set from ASL_SCORE_GROUP at create time (0: default phase grouping)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
   std::vector<AslReq> req;

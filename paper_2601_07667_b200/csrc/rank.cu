@@ -470,7 +470,8 @@ asl_status rank_static_setup(int device, RankStaticScratch** out) {
     else if (cudaGetSymbolAddress(&p, g_rank_static) != cudaSuccess || !p) st = ASL_ERR_CUDA;
     d.ptr[device] = static_cast<RankStaticScratch*>(p);
     d.status[device] = st;
-    d.done[device] = true;
+    d.done[device] = st == ASL_OK || st == ASL_ERR_ARCH;     // a failed CUDA call is tried again by the next call
+    if (st == ASL_ERR_CUDA) cudaGetLastError();
   }
   *out = d.ptr[device];
   return d.status[device];

@@ -182,7 +182,7 @@ __global__ void offsets_to_lse(const float* __restrict__ offsets, float* __restr
 // [b][h][g*W + t] and [b][h*G + g][t] are the same linear order: contiguous groups.
 asl_status asl_launch_window_lse(asl_ctx* c, const char* ws, float* lse_out, cudaStream_t st) {
   const int n = c->p.batch * c->p.n_kv_heads * c->rows_per_kv;
-  const int stride = (c->tc.enabled && !c->force_simt) ? c->tc.nchunk * c->tc.NC : c->rows_per_kv;
+  const int stride = c->tc.enabled ? c->tc.nchunk * c->tc.NC : c->rows_per_kv;
   offsets_to_lse<<<(n + 255) / 256, 256, 0, st>>>(reinterpret_cast<const float*>(ws + c->ws.score_offsets), lse_out, n,
                                                   c->rows_per_kv, stride);
   c->launches += 1;

@@ -833,8 +833,8 @@ bool asl_tc_plan(asl_ctx* c) {
   tp.nseg = (int)segs.size();
   // Segments per group: pass 1 of all of them runs before their pass 2, which hides the fold of the
   // row denominators; K of a whole group has to stay in L2 between the passes (72 MB of the 126 MB).
-  int group = c->score_group;
-  if (group <= 0) {
+  int group = 0;
+  {
     const double seg_bytes = (double)c->sum_tokens * p.k_stride[0] * 2.0 / p.n_kv_heads / (double)p.batch;   // one kv head of an average request
     group = (int)(72.0e6 / (seg_bytes > 1.0 ? seg_bytes : 1.0));
     group = group < 1 ? 1 : (group > 16 ? 16 : group);

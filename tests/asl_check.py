@@ -11,12 +11,21 @@ from paper_2601_07667_b200 import inputs as I
 SCORE_RTOL, SCORE_ATOL = 2e-3, 1e-5          # tolerance of the scores against the fp64 oracle
 
 
-def make_path(wl, device=0):
+def make_path(wl, device=0, **launch):
+    """LayerPath of a workload.  ``launch``: the launch configuration (``score_ctas``, ``tail_streams``) and
+    non-default strides (``q_stride``, ``k_stride``, ``v_stride``); omitted = the library's defaults."""
     from paper_2601_07667_b200 import binding
     return binding.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
                              window=wl.window, pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode,
                              seqlens=wl.seqlens, budgets=wl.budgets, l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau,
-                             device=device)
+                             device=device, **launch)
+
+
+def bench_launch(device=0):
+    """The launch configuration bench.py times by default: the persistent scorer on all but 16 SMs,
+    the rest of the layer on two side streams."""
+    import bench
+    return bench.default_launch(torch.cuda.get_device_properties(device).multi_processor_count)
 
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
@@ -77,12 +86,18 @@ def check_topk_against_oracle(idx_gpu: np.ndarray, ref_scores: np.ndarray, k: in
 def check_layer(path, wl, x, layer_idx, *, q_dev=None, k_dev=None, v_dev=None, ref=None, check_stat=True):
     """Runs one layer on the GPU and checks a1..a5 against the oracle.  Returns
     a dict with the GPU's aggregate (fp64) and statistic record(s)."""
-    cu = wl.cu_seqlens()
     q_dev = to_dev(x["q_obs"]) if q_dev is None else q_dev
     k_dev = to_dev(x["k"]) if k_dev is None else k_dev
     v_dev = to_dev(x["v"]) if v_dev is None else v_dev
     path.run_layer(q_dev, k_dev, v_dev, layer_idx)
     torch.cuda.synchronize()
+    return verify_layer(path, wl, x, layer_idx, ref=ref, check_stat=check_stat)
+
+
+def verify_layer(path, wl, x, layer_idx, *, ref=None, check_stat=True):
+    """Checks what the path's buffers hold after layer ``layer_idx`` (however it was issued: call by
+    call or replayed from a CUDA graph) against the oracle on the host inputs ``x``."""
+    cu = wl.cu_seqlens()
     P_gpu = path.scores_kv.cpu().numpy()
     agg_gpu = path.scores_agg.cpu().numpy()
     idx_gpu = path.idx.cpu().numpy()

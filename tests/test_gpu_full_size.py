@@ -1,13 +1,16 @@
-"""GPU parity at the benchmark's full sizes (the five named workloads), in the
-launch configuration bench.py times.  The oracle computes whole layers here
-(seconds each on the host), so the comparison stays element by element; the
-number of layers is bounded to keep the suite within minutes."""
+"""GPU parity at the benchmark's full sizes (the five named workloads).  The sweeps run in the
+library's default launch configuration (one scorer CTA per SM, one side stream); the
+``benched_launch`` tests repeat the long-context and the ragged workload in the configuration
+bench.py times (fewer scorer CTAs, two side streams), issued call by call and replayed from CUDA
+graphs.  The oracle computes whole layers here (seconds each on the host), so the comparison stays
+element by element; the number of layers is bounded to keep the suite within minutes."""
 import numpy as np
 import pytest
+import torch
 
 from paper_2601_07667_b200 import inputs as I
 
-from asl_check import StatReplay, check_layer, make_path
+from asl_check import StatReplay, bench_launch, check_layer, make_path, oracle_layer, to_dev, verify_layer
 
 pytestmark = pytest.mark.gpu
 
@@ -63,3 +66,52 @@ def test_half_million_token_context():
     wl = I.workload("C3", n_q_heads=8, n_kv_heads=2, seqlens=(524288 + 64,), budgets=(8192,), layers=2, l_min=1,
                     l_obs=2)
     sweep(wl, 3, range(0, 2))
+
+
+def _benched_launch_case(wl, seed, n_layers):
+    """Layers 0..n_layers-1 in bench.py's launch configuration: call by call, then the same layers
+    recorded one per CUDA graph and replayed twice over, every output checked against the oracle
+    after each replay."""
+    path = make_path(wl, **bench_launch())
+    xs = [I.layer_inputs(wl, l, seed) for l in range(n_layers)]
+    refs = [oracle_layer(wl, x) for x in xs]
+    dev = [(to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])) for x in xs]
+    for l in range(n_layers):                                            # (a) call by call
+        check_layer(path, wl, xs[l], l, q_dev=dev[l][0], k_dev=dev[l][1], v_dev=dev[l][2], ref=refs[l])
+    graphs, cur = [], []
+    for l in range(n_layers):                                            # (b) one layer per graph
+        graphs.append(path.capture([dev[l] + (l,)]))
+        cur.append(path._cur)                                            # score buffer the recorded layer writes
+    for _ in range(2):
+        for l in range(n_layers):
+            graphs[l].replay()
+            torch.cuda.synchronize()
+            path._cur = cur[l]
+            verify_layer(path, wl, xs[l], l, ref=refs[l])
+    from paper_2601_07667_b200 import binding as B
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
+def test_c3_benched_launch_calls_and_graph_replay():
+    _benched_launch_case(I.workload("C3"), 0, 2)
+
+
+def test_c4_benched_launch_calls_and_graph_replay():
+    _benched_launch_case(I.workload("C4", seed=0), 0, 1)
+
+
+def test_whole_bench_sequence_as_one_graph_matches_the_oracle_on_its_last_layer():
+    """The form bench.py replays: several layers, side streams included, in ONE graph."""
+    wl = I.workload("C3")
+    path = make_path(wl, **bench_launch())
+    xs = [I.layer_inputs(wl, l, 0) for l in range(3)]
+    dev = [(to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])) for x in xs]
+    for l in range(3):
+        path.run_layer(*dev[l], l)
+    graph = path.capture([dev[l] + (l,) for l in range(3)])
+    for _ in range(2):
+        graph.replay()
+        torch.cuda.synchronize()
+        verify_layer(path, wl, xs[2], 2)
+    path.close()

@@ -92,6 +92,43 @@ def test_scorer_shapes(Hq, Hk, w, mode, n):
     run_stack(wl, seed=5)
 
 
+@pytest.mark.parametrize("ctas", [100, 37, 1])
+def test_scorer_grid_sizes_that_do_not_divide_the_work(ctas):
+    """Tiles, rows to fold and publish counts are dealt by CTA index modulo the grid: odd and tiny grids."""
+    wl = I.workload("C3", seqlens=(128 * 45 + 17,), budgets=(300,), layers=2, l_min=1, l_obs=2)
+    path = make_path(wl, score_ctas=ctas, tail_streams=2)
+    for layer in range(2):
+        check_layer(path, wl, I.layer_inputs(wl, layer, 4), layer)
+    path.close()
+
+
+def _strided_case(wl, seed):
+    """K and V interleaved in one buffer (token stride 2*H_k*d, V behind K) and q_obs rows padded to 1.5 d."""
+    Hq, Hk, d, w = wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.window
+    qs = (Hq * w * (d + d // 2) + 64, w * (d + d // 2), d + d // 2)
+    ks = (2 * Hk * d, d)
+    path = make_path(wl, q_stride=qs, k_stride=ks, v_stride=ks)
+    for layer in range(2):
+        x = I.layer_inputs(wl, layer, seed)
+        n = x["k"].shape[0]
+        kv = torch.full((n, 2, Hk, d), -3.0, dtype=torch.bfloat16, device="cuda")
+        kv[:, 0] = to_dev(x["k"])
+        kv[:, 1] = to_dev(x["v"])
+        qbuf = torch.full((wl.batch * qs[0],), 7.0, dtype=torch.bfloat16, device="cuda")
+        qv = torch.as_strided(qbuf, (wl.batch, Hq, w, d), qs + (1,))
+        qv.copy_(to_dev(x["q_obs"]))
+        check_layer(path, wl, x, layer, q_dev=qv, k_dev=kv[:, 0], v_dev=kv[:, 1])
+    path.close()
+
+
+def test_strided_inputs_on_the_tensor_core_scorer():
+    _strided_case(I.workload("C3", seqlens=(2900,), budgets=(400,), layers=2, l_min=1, l_obs=2), 6)
+
+
+def test_strided_inputs_on_the_cuda_core_scorer():
+    _strided_case(I.workload("C1", seqlens=(1500, 700), budgets=(200, 100), window=24, layers=2, l_min=1, l_obs=2), 6)
+
+
 def test_logits_far_above_the_first_keys_of_a_row():
     """Keys whose logit exceeds the row's reference (the maximum over its first 32 keys) by more than
     fp32's exponent range, so that the plain pass-1 sums overflow: in the last 32 keys of a tile (redone

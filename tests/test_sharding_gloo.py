@@ -57,6 +57,31 @@ def test_two_ranks_shard_requests_and_reduce_the_slowest_time(tmp_path):
     assert value[0] == pytest.approx(2 * 600 / 2.0e-3)                   # whole-job tokens / slowest time
 
 
+def test_bench_started_without_a_launcher_spawns_its_own_ranks():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment: the script starts the two
+    replicas itself; rank 0 prints one line for the whole job (here without kernels, gloo on CPU)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--seed", "5"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, "one line for the whole job, from rank 0"
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 2.0          # slowest rank's time
+    assert lines[0]["seed_of_last_rank"] == 6                                    # ranks draw their own requests
+    assert lines[0]["value"] == pytest.approx(2 * 1000 / 2.0e-3)
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1", MASTER_PORT="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--dry-run"], env=env,
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "WORLD_SIZE" in r.stderr
+
+
 def test_single_rank_helpers_need_no_process_group():
     sys.path.insert(0, ROOT)
     import bench
