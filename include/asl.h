@@ -25,6 +25,16 @@
  *     disjoint regions per entry point, so asl_rank_stat may run on another
  *     stream concurrently with asl_select_topk / asl_compact_kv of the same
  *     layer.  Two calls of the SAME entry point on one context must not overlap.
+ *   - At most ONE scoring call (asl_score_layer, asl_score_layer_lse,
+ *     asl_score_columns) may be in flight per DEVICE, whatever the context,
+ *     stream or process: the scorer is one persistent kernel whose CTAs wait for
+ *     one another, so all of them have to be resident at the same time.  Its grid
+ *     never exceeds the SM count and one CTA fills an SM, which makes that true
+ *     when it has the SMs it asks for; two scorers started side by side could each
+ *     hold part of the SMs and wait for CTAs that cannot start.  Such a wait is
+ *     bounded (2 s) and ends in ASL_ERR_TIMEOUT, never in a hang, but the results
+ *     of both calls are then void.  Order scoring calls of different contexts on
+ *     one device with events.  Every other entry point may overlap freely.
  *   - bf16 tensors are passed as raw 16-bit patterns; the channel (head_dim)
  *     axis is contiguous and every row starts on a 16-byte boundary.
  *   - Token indices are request-local, 0-based, int32.
@@ -241,6 +251,17 @@ asl_status asl_rank_desc_static(const float* scores, int32_t T, int32_t* rank_ou
  * it waits for `stream` first).  ASL_OK, or ASL_ERR_TIMEOUT with *where set to
  * the code of the wait that gave up; the word is cleared. */
 asl_status asl_device_status(asl_ctx* ctx, void* stream, int32_t* where);
+
+/* Self-test of the bounded waits (no counterpart in the paper: a diagnostic of this library).  The
+ * scorer's kernels wait on shared-memory barriers and on counters in device memory; every such wait
+ * gives up after a time limit, records a code in the context's error word and lets the kernel finish,
+ * so that a wait that can never end surfaces as ASL_ERR_TIMEOUT instead of a hung device.  This call
+ * launches one warp that runs one of those two waits -- which = 0: a barrier nobody arrives on;
+ * which = 1: a counter nobody advances -- with the limit `limit_ns` (1 us .. 1 ms), so the path can be
+ * exercised without any fault: afterwards asl_device_status returns ASL_ERR_TIMEOUT with *where = 91
+ * (barrier) or 92 (counter), and the query after that ASL_OK.  Needs a planned context; asynchronous
+ * on `stream`. */
+asl_status asl_selftest_bounded_wait(asl_ctx* ctx, int32_t which, int64_t limit_ns, void* stream);
 
 /* Number of kernels this context has launched so far (host counter). */
 int64_t asl_launch_count(const asl_ctx* ctx);

@@ -20,7 +20,8 @@ ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score_layer", "asl_rank_stat",
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
            "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows",
-           "asl_score_columns", "asl_pool_scores", "asl_set_controller", "asl_select_topk_gated")
+           "asl_score_columns", "asl_pool_scores", "asl_set_controller", "asl_select_topk_gated",
+           "asl_selftest_bounded_wait")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -75,6 +76,7 @@ def _load() -> C.CDLL:
     lib.asl_compact_kv.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.asl_device_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.asl_rank_desc_static.argtypes = [vp, i32, vp, vp]
+    lib.asl_selftest_bounded_wait.argtypes = [vp, i32, i64, vp]
     lib.asl_launch_count.argtypes = [vp]
     lib.asl_launch_count.restype = i64
     lib.asl_strerror.argtypes = [C.c_int]
@@ -214,6 +216,11 @@ def asl_device_status(ctx, stream=None):
     where = C.c_int32(0)
     st = _lib.asl_device_status(ctx, _stream_handle(stream), C.byref(where))
     return st, where.value
+
+
+def asl_selftest_bounded_wait(ctx, which: int, limit_ns: int, stream=None) -> None:
+    _check(_lib.asl_selftest_bounded_wait(ctx, int(which), int(limit_ns), _stream_handle(stream)),
+           "asl_selftest_bounded_wait")
 
 
 def asl_launch_count(ctx) -> int:

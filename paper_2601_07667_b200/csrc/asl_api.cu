@@ -271,6 +271,11 @@ asl_status asl_device_status(asl_ctx* c, void* stream, int32_t* where) {
   return ASL_ERR_TIMEOUT;
 }
 
+asl_status asl_selftest_bounded_wait(asl_ctx* c, int32_t which, int64_t limit_ns, void* stream) {
+  if (!c || !c->planned || (which != 0 && which != 1) || limit_ns < 1000 || limit_ns > 1000000) return ASL_ERR_INVALID;
+  return asl_launch_wait_selftest(c, which, (unsigned long long)limit_ns, static_cast<cudaStream_t>(stream));
+}
+
 int64_t asl_launch_count(const asl_ctx* c) { return c ? c->launches : 0; }
 
 const char* asl_strerror(asl_status s) {

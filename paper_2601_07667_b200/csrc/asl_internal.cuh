@@ -75,6 +75,7 @@ bool asl_tc_plan(asl_ctx* c);
 void asl_tc_free(asl_ctx* c);
 size_t asl_tc_partial_bytes(const asl_ctx* c);
 asl_status asl_tc_reset_sync(asl_ctx* c, cudaStream_t st);
+asl_status asl_launch_wait_selftest(asl_ctx* c, int which, unsigned long long limit_ns, cudaStream_t st);
 asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
                                cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);

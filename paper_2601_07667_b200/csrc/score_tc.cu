@@ -94,7 +94,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait.  `watch_abort`: also give up when another role raised the flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code,
-                                          bool watch_abort) {
+                                          bool watch_abort, unsigned long long limit_ns = WAIT_LIMIT_NS) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
@@ -102,7 +102,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (watch_abort && *abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) break;
+      else if (now - t0 > limit_ns) break;
     }
   }
   *abort_flag = code;
@@ -110,7 +110,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 // Bounded wait until the 32-bit word at p equals `want` (acquire).  Lane 0 polls.
 __device__ __forceinline__ bool word_wait(const uint32_t* p, uint32_t want, volatile int* abort_flag, int code, int lane,
-                                          uint32_t nap_max) {
+                                          uint32_t nap_max, unsigned long long limit_ns = WAIT_LIMIT_NS) {
   int gave_up = 0;
   if (lane == 0) {
     unsigned long long t0 = 0;
@@ -122,7 +122,7 @@ __device__ __forceinline__ bool word_wait(const uint32_t* p, uint32_t want, vola
       if ((it & 7u) == 7u) {
         const unsigned long long now = global_ns();
         if (t0 == 0) t0 = now;
-        else if (now - t0 > WAIT_LIMIT_NS || *abort_flag) { gave_up = 1; if (!*abort_flag) *abort_flag = code; break; }
+        else if (now - t0 > limit_ns || *abort_flag) { gave_up = 1; if (!*abort_flag) *abort_flag = code; break; }
       }
       __nanosleep(nap);
       if (nap < nap_max) nap <<= 1;
@@ -765,6 +765,27 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
 }
 
+// One warp runs one of the kernel's two kinds of bounded wait on something that never happens (a barrier
+// nobody arrives on, a counter nobody advances) with a short limit, and reports like the scorer does.
+__global__ void bounded_wait_selftest_kernel(int which, unsigned long long limit_ns, const uint32_t* never_written,
+                                             int32_t* err) {
+  __shared__ __align__(8) unsigned long long s_bar;
+  __shared__ int s_flag;
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&s_bar), 1);
+    s_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &s_flag;
+  bool ok;
+  if (which == 0) ok = mbar_wait(smem_u32(&s_bar), 0, abort_flag, 91, true, limit_ns);
+  else            ok = word_wait(never_written, 0xFFFFFFFFu, abort_flag, 92, lane, 256, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && !ok && *abort_flag) atomicCAS(err, 0, *abort_flag);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -896,6 +917,13 @@ void asl_tc_free(asl_ctx* c) {
   tp.d_phases2 = nullptr;
   tp.d_sync = nullptr;
   tp.enabled = false;
+}
+
+asl_status asl_launch_wait_selftest(asl_ctx* c, int which, unsigned long long limit_ns, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(which, limit_ns, reinterpret_cast<const uint32_t*>(c->d_err), c->d_err);   // the error word is never all ones
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
 }
 
 // after a reported device error the publish counters may be inconsistent: start over

@@ -68,6 +68,14 @@ def test_half_million_token_context():
     sweep(wl, 3, range(0, 2))
 
 
+def test_million_token_context():
+    """1048640 tokens in one request (8q/2kv): 8193 key tiles per segment, 512 rank tiles, 256 top-k tiles;
+    score and token offsets beyond 2^20, packed K rows beyond 2^31 bytes."""
+    wl = I.workload("C3", n_q_heads=8, n_kv_heads=2, seqlens=(1048576 + 64,), budgets=(8192,), layers=1, l_min=1,
+                    l_obs=2)
+    sweep(wl, 4, range(0, 1))
+
+
 def _benched_launch_case(wl, seed, n_layers):
     """Layers 0..n_layers-1 in bench.py's launch configuration: call by call, then the same layers
     recorded one per CUDA graph and replayed twice over, every output checked against the oracle

@@ -129,6 +129,26 @@ def test_strided_inputs_on_the_cuda_core_scorer():
     _strided_case(I.workload("C1", seqlens=(1500, 700), budgets=(200, 100), window=24, layers=2, l_min=1, l_obs=2), 6)
 
 
+@pytest.mark.parametrize("which,code", [(0, 91), (1, 92)])
+def test_a_wait_that_cannot_end_surfaces_as_a_timeout_status(which, code):
+    """The scorer's waits are bounded.  One warp waits 20 us on a barrier nobody arrives on / a counter
+    nobody advances: the kernel returns by itself, the context reports ASL_ERR_TIMEOUT with the code of
+    the wait, the report clears the error word, and the context keeps working."""
+    from paper_2601_07667_b200 import binding as B
+    wl = I.workload("C1", seqlens=(700,), budgets=(100,), layers=1)
+    path = make_path(wl)
+    assert B.asl_device_status(path.ctx) == (B.ASL_OK, 0)
+    B.asl_selftest_bounded_wait(path.ctx, which, 20000)
+    assert B.asl_device_status(path.ctx) == (B.ASL_ERR_TIMEOUT, code)
+    assert B.asl_device_status(path.ctx) == (B.ASL_OK, 0)
+    check_layer(path, wl, I.layer_inputs(wl, 0, 2), 0)                 # the context is still usable
+    with pytest.raises(B.AslError):
+        B.asl_selftest_bounded_wait(path.ctx, 2, 20000)
+    with pytest.raises(B.AslError):
+        B.asl_selftest_bounded_wait(path.ctx, 0, 10**9)                 # limits beyond 1 ms are refused
+    path.close()
+
+
 def test_logits_far_above_the_first_keys_of_a_row():
     """Keys whose logit exceeds the row's reference (the maximum over its first 32 keys) by more than
     fp32's exponent range, so that the plain pass-1 sums overflow: in the last 32 keys of a tile (redone
