@@ -30,9 +30,20 @@ from paper_2601_07667_b200 import inputs as I   # noqa: E402
 
 METRIC = "obs-window score+select+compact: context tokens/s/layer"
 UNIT = "tokens/s/layer"
-# dram__bytes_read.sum + dram__bytes_write.sum of one scorer launch, from the ncu capture summarised in
-# profiles/score_tc_fused_c3_128k_dram_traffic.txt (set to None when the scorer changes until re-captured)
-SCORER_TRAFFIC_BYTES = {"C3": 279.4e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one scorer launch: read from the committed summary of the ncu
+# capture (its "traffic_bytes_per_launch:" line), so that the figure and the evidence cannot drift apart
+SCORER_TRAFFIC_FILES = {"C3": os.path.join(ROOT, "profiles", "score_tc_kernel_c3_128k_dram_traffic.txt")}
+
+
+def scorer_traffic_bytes(workload_name):
+    path = SCORER_TRAFFIC_FILES.get(workload_name)
+    if not path or not os.path.exists(path):
+        return None
+    with open(path) as f:
+        for line in f:
+            if line.startswith("traffic_bytes_per_launch:"):
+                return float(line.split(":")[1])
+    return None
 # default launch configuration of the timed steps (the GPU parity tests build their paths from the same two values)
 DEFAULT_SCORE_CTAS = -16       # persistent scorer: this many CTAs fewer than SMs (0 = one per SM)
 DEFAULT_TAIL_STREAMS = 2       # side streams for the rest of the layer
@@ -485,7 +496,7 @@ def run_ours(args):
         achieved = work["flops"] / (score_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": tf, "unit": "TFLOP/s", "frac": achieved / tf}
     default_shape = not args.seqlens and not args.budgets and not args.heads
-    roof.update({"traffic": SCORER_TRAFFIC_BYTES.get(wl.name) if default_shape else None, "kernel": "score_tc_kernel (asl_score_columns: both softmax passes, one persistent launch)", "kernel_ms": score_ms,
+    roof.update({"traffic": scorer_traffic_bytes(wl.name) if default_shape else None, "kernel": "score_tc_kernel (asl_score_columns: both softmax passes, one persistent launch)", "kernel_ms": score_ms,
                  "peak_source": pk["source"], "step_roofline_us": max(t_hbm, t_mma) * 1e6,
                  "step_frac": max(t_hbm, t_mma) / (ms_step * 1e-3)})
 

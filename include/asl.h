@@ -188,9 +188,24 @@ asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, i
  * asl_select_topk_gated is asl_select_topk for the requests whose record (`stat`, device [B], as written by
  * the asl_rank_stat call of layer `layer_idx` ordered before it) selected at exactly that layer; the lists of
  * all other requests are left untouched.  With n_heads = 1 on scores_agg, called after every layer's
- * asl_rank_stat, it leaves in idx_out the one-shot selection of Algorithm 2 for every request that selected. */
+ * asl_rank_stat, it leaves in idx_out the one-shot selection of Algorithm 2 for every request that selected.
+ *
+ * Under ASL_CONTROLLER_LATCH the work of a finished request is skipped as well (Algorithm 2 ends the
+ * method for a request at its selection layer: only select_idx goes on and the rank cache is released).
+ * A request is finished at layer l when its record selected at a layer before l.  asl_set_layer tells
+ * the context which layer the calls that follow belong to (call it at the start of every layer); the
+ * records consulted are those passed to the latest asl_rank_stat call.  Then, for a finished request,
+ *   - the scorer leaves out its phases (the flags are read once, ahead of the launch, so a record that a
+ *     still-running asl_rank_stat of the previous layer is about to set takes effect one layer later);
+ *   - asl_pool_scores, asl_select_topk and asl_compact_kv leave its scores, kept list and compacted
+ *     cache as its selection layer wrote them; they read the records on the device, so issue them after
+ *     (on the same stream as, or ordered behind) the asl_rank_stat call of the previous layer;
+ *   - its rows of the rank ring are dead: nothing reads or writes them again, the caller may reuse them.
+ * Batches of more than 256 requests are scored in full (the other calls still skip).  Without
+ * asl_set_layer (or in ASL_CONTROLLER_REPORT) nothing is skipped. */
 enum { ASL_CONTROLLER_REPORT = 0, ASL_CONTROLLER_LATCH = 1 };
 asl_status asl_set_controller(asl_ctx* ctx, int32_t mode);
+asl_status asl_set_layer(asl_ctx* ctx, int32_t layer_idx);
 asl_status asl_select_topk_gated(asl_ctx* ctx, const float* scores, int32_t n_heads, int32_t* idx_out,
                                  const asl_stat* stat, int32_t layer_idx, void* workspace, size_t workspace_bytes,
                                  void* stream);

@@ -21,7 +21,7 @@ EXPORTS = ("asl_create", "asl_destroy", "asl_plan", "asl_plan_sizes", "asl_score
            "asl_select_topk", "asl_compact_kv", "asl_device_status", "asl_launch_count", "asl_strerror",
            "asl_rank_desc_static", "asl_score_layer_lse", "asl_window_lse", "asl_compact_rows",
            "asl_score_columns", "asl_pool_scores", "asl_set_controller", "asl_select_topk_gated",
-           "asl_selftest_bounded_wait")
+           "asl_selftest_bounded_wait", "asl_set_layer")
 ASL_RANK_STATIC_MAX_T = 262144
 
 
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
     lib.asl_score_layer_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.asl_window_lse.argtypes = [vp, vp, sz, vp, vp]
     lib.asl_set_controller.argtypes = [vp, i32]
+    lib.asl_set_layer.argtypes = [vp, i32]
     lib.asl_select_topk_gated.argtypes = [vp, vp, i32, vp, vp, i32, vp, sz, vp]
     lib.asl_score_columns.argtypes = [vp, vp, vp, vp, vp, sz, i32, vp]
     lib.asl_pool_scores.argtypes = [vp, vp, sz, i32, vp, vp, vp]
@@ -169,6 +170,10 @@ ASL_CONTROLLER_REPORT, ASL_CONTROLLER_LATCH = 0, 1
 
 def asl_set_controller(ctx, mode: int) -> None:
     _check(_lib.asl_set_controller(ctx, int(mode)), "asl_set_controller")
+
+
+def asl_set_layer(ctx, layer_idx: int) -> None:
+    _check(_lib.asl_set_layer(ctx, int(layer_idx)), "asl_set_layer")
 
 
 def asl_select_topk_gated(ctx, scores, n_heads, idx_out, stat, layer_idx, workspace, workspace_bytes, stream=None) -> None:
@@ -291,6 +296,13 @@ class LayerPath:
         self._join = torch.cuda.Event()
         self._join2 = torch.cuda.Event()
         self.first_layer: Optional[int] = None
+        self.latch = False
+
+    def set_controller(self, mode: int) -> None:
+        """ASL_CONTROLLER_LATCH: selections are final on the device and ``run_layer`` tells the library the
+        layer of its calls, so that the work of finished requests is skipped."""
+        asl_set_controller(self.ctx, mode)
+        self.latch = mode == ASL_CONTROLLER_LATCH
 
     @property
     def scores_kv(self):
@@ -363,6 +375,8 @@ class LayerPath:
         ctx, ws, wsb = self.ctx, self.workspace, self.ws_bytes
         rows = self.n_rows(layer_idx)
         main = torch.cuda.current_stream()
+        if self.latch:
+            asl_set_layer(ctx, layer_idx)
         self._cur ^= 1
         agg, skv = self._agg[self._cur], self._kv[self._cur]
         if self._agg_free[self._cur] is not None:

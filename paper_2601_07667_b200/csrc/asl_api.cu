@@ -13,8 +13,12 @@ void free_plan(asl_ctx* c) {
   asl_tc_free(c);
   if (c->d_req) cudaFree(c->d_req);
   if (c->d_acc) cudaFree(c->d_acc);
+  if (c->d_skip) cudaFree(c->d_skip);
   c->d_req = nullptr;
   c->d_acc = nullptr;
+  c->d_skip = nullptr;
+  c->latch_stat = nullptr;
+  c->cur_layer = -1;
   c->planned = false;
 }
 
@@ -106,6 +110,8 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   if (e == cudaSuccess) e = cudaMemcpy(c->d_req, req.data(), sizeof(AslReq) * p->batch, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&c->d_acc, sizeof(unsigned long long) * (2 * p->batch + 1));
   if (e == cudaSuccess) e = cudaMemset(c->d_acc, 0, sizeof(unsigned long long) * (2 * p->batch + 1));
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_skip, sizeof(uint32_t) * (ASL_SKIP_MAX_BATCH / 32));
+  if (e == cudaSuccess) e = cudaMemset(c->d_skip, 0, sizeof(uint32_t) * (ASL_SKIP_MAX_BATCH / 32));
   cudaSetDevice(prev);
   if (e != cudaSuccess) { free_plan(c); return ASL_ERR_CUDA; }
 
@@ -171,7 +177,15 @@ static asl_status score_columns_impl(asl_ctx* c, const void* q_obs, const void* 
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
   float* u = reinterpret_cast<float*>(ws + c->ws.score_u[slot]);
-  if (c->tc.enabled) return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
+  if (c->tc.enabled) {
+    // requests that have finished are not scored any more: their flags are read once, ahead of the launch,
+    // so that every CTA of the persistent kernel leaves out the same phases
+    if (c->latch_stat && c->cur_layer >= 0 && c->p.batch <= ASL_SKIP_MAX_BATCH) {
+      const asl_status s = asl_launch_skip_snapshot(c, static_cast<cudaStream_t>(stream));
+      if (s != ASL_OK) return s;
+    }
+    return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
+  }
   return asl_launch_score_simt(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));
 }
 
@@ -218,6 +232,7 @@ asl_status asl_rank_stat(asl_ctx* c, const float* scores_agg, int32_t layer_idx,
   if (!c || !c->planned || !scores_agg || !rank_ring || !stat) return ASL_ERR_INVALID;
   if (layer_idx < 0 || n_rows < 1 || n_rows > c->p.l_obs || n_rows > layer_idx + 1) return ASL_ERR_INVALID;
   if (!workspace || workspace_bytes < c->ws.total || !aligned16(workspace)) return ASL_ERR_WORKSPACE;
+  if (c->controller == ASL_CONTROLLER_LATCH) c->latch_stat = stat;
   return asl_launch_rank(c, scores_agg, layer_idx, n_rows, rank_ring, stat, static_cast<char*>(workspace),
                          static_cast<cudaStream_t>(stream));
 }
@@ -241,6 +256,13 @@ asl_status asl_select_topk_gated(asl_ctx* c, const float* scores, int32_t n_head
 asl_status asl_set_controller(asl_ctx* c, int32_t mode) {
   if (!c || (mode != ASL_CONTROLLER_REPORT && mode != ASL_CONTROLLER_LATCH)) return ASL_ERR_INVALID;
   c->controller = mode;
+  if (mode != ASL_CONTROLLER_LATCH) c->latch_stat = nullptr;
+  return ASL_OK;
+}
+
+asl_status asl_set_layer(asl_ctx* c, int32_t layer_idx) {
+  if (!c || layer_idx < 0) return ASL_ERR_INVALID;
+  c->cur_layer = layer_idx;
   return ASL_OK;
 }
 

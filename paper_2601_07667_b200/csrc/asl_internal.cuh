@@ -40,6 +40,9 @@ struct asl_ctx {
   int sm_count = 0;
   bool planned = false;
   int controller = 0;                 // ASL_CONTROLLER_*: asl_set_controller
+  const asl_stat* latch_stat = nullptr;   // under ASL_CONTROLLER_LATCH: the records of the latest asl_rank_stat call (device)
+  int32_t cur_layer = -1;             // layer the next calls belong to (asl_set_layer / asl_rank_stat)
+  uint32_t* d_skip = nullptr;         // device [8]: bit b set = request b finished before cur_layer (scorer's snapshot)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
   std::vector<AslReq> req;
@@ -58,6 +61,21 @@ struct asl_ctx {
   AslWorkspace ws{};
   int64_t launches = 0;
 };
+
+// Under ASL_CONTROLLER_LATCH a request is finished at layer `cur` once its record selected at an
+// earlier layer: Algorithm 2 has returned its one-shot selection and the method does nothing more for it.
+// The record may be being written by an asl_rank_stat of the same layer on another stream: the writer
+// stores `selected` last, behind a fence, and the reader looks at layer_idx only after it has seen
+// `selected`, so a record in the middle of its update reads as "not finished" or with its final layer.
+#ifdef __CUDACC__
+__device__ inline bool asl_finished(const asl_stat* s, int32_t cur) {
+  const volatile asl_stat* v = s;
+  if (!v->selected) return false;
+  __threadfence();
+  return v->layer_idx < cur;
+}
+#endif
+constexpr int ASL_SKIP_MAX_BATCH = 256;   // requests the scorer's skip mask covers (larger batches are scored in full)
 
 #define ASL_CUDA(expr)                          \
   do {                                          \
@@ -79,6 +97,7 @@ asl_status asl_launch_wait_selftest(asl_ctx* c, int which, unsigned long long li
 asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
                                cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
+asl_status asl_launch_skip_snapshot(asl_ctx* c, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);
 asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* gate,

@@ -7,9 +7,11 @@ namespace {
 __global__ void __launch_bounds__(256) compact_kv_kernel(const uint16_t* __restrict__ k, const uint16_t* __restrict__ v,
                                                          const int32_t* __restrict__ idx, const AslReq* __restrict__ req,
                                                          int64_t ks_t, int64_t ks_h, int64_t vs_t, int64_t vs_h,
-                                                         int64_t sum_kept, int vec_per_row, uint16_t* __restrict__ k_out,
+                                                         int64_t sum_kept, int vec_per_row, const asl_stat* __restrict__ latch,
+                                                         int cur_layer, uint16_t* __restrict__ k_out,
                                                          uint16_t* __restrict__ v_out) {
   const int b = blockIdx.z, h = blockIdx.y;
+  if (latch && asl_finished(latch + b, cur_layer)) return;       // finished request: its compacted cache is final
   const AslReq rq = req[b];
   const int rows_per_block = blockDim.x / vec_per_row;
   const int r = blockIdx.x * rows_per_block + threadIdx.x / vec_per_row;
@@ -58,6 +60,7 @@ asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const in
   dim3 grid((c->max_kept + rows_per_block - 1) / rows_per_block, p.n_kv_heads, p.batch);
   compact_kv_kernel<<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), idx, c->d_req,
                                           p.k_stride[0], p.k_stride[1], p.v_stride[0], p.v_stride[1], c->sum_kept, vec,
+                                          c->latch_stat, c->cur_layer,
                                           static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out));
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());

@@ -26,9 +26,11 @@ constexpr int HB = 8;            // staged rows per round: their loads are all i
 // over all heads in a fixed order: no atomics, bit-reproducible.
 __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
                                                         int Hk, int G, int S, int mode, int urows, int parts, int64_t sum_T,
+                                                        const asl_stat* __restrict__ latch, int cur_layer,
                                                         float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
   __shared__ float tile[HB][PT + 2 * MAX_HALO];
   const int b = blockIdx.y;
+  if (latch && asl_finished(latch + b, cur_layer)) return;      // the request's scores stay as its selection layer left them
   const AslReq rq = req[b];
   const int j0 = blockIdx.x * PT;
   if (j0 >= rq.T) return;
@@ -85,14 +87,30 @@ __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict_
   if (live) scores_agg[rq.t_off + j] = agg;
 }
 
+// bit b of mask[b / 32]: request b has finished before layer `cur` (read by the scorer launched next)
+__global__ void skip_snapshot_kernel(const asl_stat* __restrict__ latch, int cur, int batch, uint32_t* __restrict__ mask) {
+  const int b = threadIdx.x;
+  const bool fin = b < batch && asl_finished(latch + b, cur);
+  const uint32_t word = __ballot_sync(0xffffffffu, fin);
+  if ((b & 31) == 0) mask[b >> 5] = word;
+}
+
 }  // namespace
+
+asl_status asl_launch_skip_snapshot(asl_ctx* c, cudaStream_t st) {
+  skip_snapshot_kernel<<<1, ASL_SKIP_MAX_BATCH, 0, st>>>(c->latch_stat, c->cur_layer, c->p.batch, c->d_skip);
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}
 
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st) {
   const asl_params& p = c->p;
   if (p.pool_kernel / 2 > MAX_HALO) return ASL_ERR_UNSUPPORTED;
   dim3 grid((c->max_T + PT - 1) / PT, p.batch);
   pool_group_kernel<<<grid, PT, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
-                                          p.pool_mode, c->u_rows_per_kv, c->u_parts, c->sum_T, scores_kv, scores_agg);
+                                          p.pool_mode, c->u_rows_per_kv, c->u_parts, c->sum_T, c->latch_stat, c->cur_layer,
+                                          scores_kv, scores_agg);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

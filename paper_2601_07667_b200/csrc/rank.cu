@@ -316,7 +316,13 @@ __device__ void stat_finalize_one(unsigned long long* acc, const AslReq* __restr
     s.rel = s.var_top / s.init_var;
     s.selected = (s.rel < tau) ? 1 : 0;
   }
+  const int32_t selected = s.selected;
+  s.selected = 0;
   stat[b] = s;
+  if (selected) {                                      // last, behind a fence: see asl_finished
+    __threadfence();
+    reinterpret_cast<volatile asl_stat*>(stat + b)->selected = 1;
+  }
 }
 
 // layers before L_min (or with a single rank row): only the bookkeeping fields change

@@ -304,6 +304,7 @@ struct TcArgs {
   uint32_t* folded;        // [segment] rows whose offset is written, accumulated over launches
   int32_t* err;
   int64_t sum_T;
+  const uint32_t* skip_mask;   // null, or bit b set: request b has finished (device-side controller): its phases are left out
   uint32_t* epoch_word;    // two-pass launches completed so far (the counters accumulate over launches); then a ticket word
   uint32_t epoch_limit;    // beyond it the last CTA clears the counters instead of letting them wrap
   int32_t nseg;
@@ -350,6 +351,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM_MISC + 4);
   volatile uint32_t* s_epoch = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC + 8);
+  volatile uint32_t* s_skip = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC + 16);   // [8]: the launch's copy of the skip mask
+  // every role leaves out the same phases: the item numbering below counts live items only
+  auto skipped = [&](int b) { return b < ASL_SKIP_MAX_BATCH && ((s_skip[b >> 5] >> (b & 31)) & 1u) != 0u; };
   float* s_negoff = reinterpret_cast<float*>(smem + SM_NEGOFF);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = a.NC;
@@ -358,6 +362,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // ---- set-up: zero the Q buffers (rows past NC feed unused MMA rows), barriers, tensor memory ----
   if (NC & 127)
     for (int i = threadIdx.x; i < 2 * Q_BUF_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
+  if (threadIdx.x >= 32 && threadIdx.x < 32 + ASL_SKIP_MAX_BATCH / 32)
+    s_skip[threadIdx.x - 32] = a.skip_mask ? __ldcg(a.skip_mask + (threadIdx.x - 32)) : 0u;
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(BAR_FULL + s), 1); mbar_init(bar(BAR_EMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
@@ -419,21 +425,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         q_issued = l;
         return true;
       };
-      for (; ok && w.valid(); w.next(), ++item) {
+      for (; ok && w.valid(); w.next()) {
         const TcPhase p = w.phase();
+        if (skipped(p.b)) continue;
         if (w.ph != cur_ph) {
           cur_ph = w.ph;
           ++lp;
           tok_off = p.tok_off;
           if (q_issued < lp && !issue_q(lp, p, true)) { ok = false; break; }
-          // where does this CTA go after this phase?
-          const int end = p.g0 + p.ntiles;
-          const int gn = w.g + ((end - w.g + (int)gridDim.x - 1) / (int)gridDim.x) * (int)gridDim.x;
+          // where does this CTA go after this phase?  (the next phase in which it has a tile and that is not left out)
+          const int grid = (int)gridDim.x;
+          int gn = w.g + ((p.g0 + p.ntiles - w.g + grid - 1) / grid) * grid;
+          int q = w.ph + 1;
           next_ph = -1;
-          if (gn < a.total_items) {
-            int q = w.ph + 1;
+          while (gn < a.total_items) {
             while (gn >= a.phases[q].g0 + a.phases[q].ntiles) ++q;
-            next_ph = q;
+            if (!skipped(a.phases[q].b)) { next_ph = q; break; }
+            gn += ((a.phases[q].g0 + a.phases[q].ntiles - gn + grid - 1) / grid) * grid;
           }
         }
         if (next_ph >= 0 && q_issued == lp) {    // prefetch the next phase's Q chunk once its buffer is free
@@ -447,6 +455,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint64_t pol = p.pass == 1 ? pol_keep : pol_stream;
         tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok, pol);
         tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok, pol);
+        ++item;
       }
       if (!ok) {
         // let the copies already issued land before the CTA's shared memory is released
@@ -468,8 +477,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t idesc1 = instr_desc(128, KT), idesc2 = instr_desc(KT, NC);
       const int nhalf = (NC > 128) ? 2 : 1;
       uint32_t qbase = 0;
-      for (; ok && w.valid(); w.next(), ++item) {
+      for (; ok && w.valid(); w.next()) {
         const TcPhase p = w.phase();
+        if (skipped(p.b)) continue;
         if (w.ph != cur_ph) {
           cur_ph = w.ph;
           ++lp;
@@ -502,6 +512,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_commit(bar(BAR_EMPTY + s));       // smem stage free once these MMAs have read it
         tc_commit(bar(BAR_TFULL + acc));     // accumulator ready for the epilogue
         if (w.last_in_phase()) tc_commit(bar(BAR_QEMPTY + (lp & 1)));   // last tile of the phase here
+        ++item;
       }
       if (!ok) {  // make sure nothing is still writing tensor memory before it is freed
         tc_commit(bar(BAR_DRAIN));
@@ -518,7 +529,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int entries = 2 * grid;                                  // entry e: CTA e/2, set e%2
     for (int ph = 0; ph < a.n_phases; ++ph) {
       const TcPhase p = a.phases[ph];
-      if (p.pass != 1) continue;
+      if (p.pass != 1 || skipped(p.b)) continue;
       if ((int)blockIdx.x + hw * grid >= NC) continue;             // no row of this segment is ours
       if (!word_wait(a.published + p.seg, epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 256)) break;
       const int first = p.g0 % grid;
@@ -583,8 +594,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // exceed 1, fp32 has the range), unless a sum overflows, in which case the tile is redone with it.
     float mref = -INFINITY, l = 0.f;
     bool first_tile = true;                 // this set has not yet taken a tile of the current pass-1 phase
-    for (; w.valid(); w.next(), ++item) {
+    for (; w.valid(); w.next()) {
       const TcPhase p = w.phase();
+      if (skipped(p.b)) continue;
       if (w.ph != cur_ph) {
         cur_ph = w.ph;
         if (p.pass == 1) {
@@ -738,6 +750,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           atomicAdd(a.published + p.seg, 1u);
         }
       }
+      ++item;
     }
   }
 
@@ -758,6 +771,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < 2 * a.nseg; ++i) a.published[i] = 0;      // published and folded are contiguous
         a.epoch_word[0] = 0;
       } else {
+        // segments that were left out: their counters advance as if they had been scored, so that a later
+        // launch that scores them again (a new prompt) finds them where its launch number expects them
+        for (int ph = 0; ph < a.n_phases; ++ph) {
+          const TcPhase q = a.phases[ph];
+          if (q.pass == 1 && skipped(q.b)) { a.published[q.seg] += 2u * (uint32_t)q.ncontrib; a.folded[q.seg] += (uint32_t)NC; }
+        }
         a.epoch_word[0] = epoch;
       }
       __threadfence();
@@ -964,6 +983,7 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   a.folded = tp.d_sync + tp.nseg;
   a.err = c->d_err;
   a.sum_T = c->sum_T;
+  a.skip_mask = (c->latch_stat && c->cur_layer >= 0 && p.batch <= ASL_SKIP_MAX_BATCH) ? c->d_skip : nullptr;
   a.epoch_word = tp.d_sync + 2 * tp.nseg;         // the one-pass launch touches neither the counters nor this
   a.epoch_limit = 0xFFFFFFFFu / (uint32_t)(2 * tp.grid > MAX_NC ? 2 * tp.grid : MAX_NC) - 2u;
   a.nseg = tp.nseg;

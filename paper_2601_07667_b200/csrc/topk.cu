@@ -42,6 +42,8 @@ struct TopkArgs {
   int32_t n_heads, max_tiles;
   const asl_stat* gate;  // null, or: only requests whose statistic selected at layer `gate_layer` are worked on
   int32_t gate_layer;
+  const asl_stat* latch; // null, or: requests that finished before layer `cur_layer` are left alone
+  int32_t cur_layer;
 };
 
 struct Segment {
@@ -60,6 +62,7 @@ __device__ __forceinline__ Segment segment_of(const TopkArgs& a) {
   const int64_t seg = (int64_t)b * a.n_heads + h;
   Segment s;
   s.open = !a.gate || (a.gate[b].selected && a.gate[b].layer_idx == a.gate_layer);
+  if (a.latch && asl_finished(a.latch + b, a.cur_layer)) s.open = false;
   s.row = a.scores + (int64_t)h * a.sum_T + rq.t_off;
   s.hist = a.scratch + seg * SEG_INTS;
   s.state = s.hist + 3 * BINS;
@@ -286,6 +289,8 @@ asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
   a.max_tiles = tiles;
   a.gate = gate;
   a.gate_layer = gate_layer;
+  a.latch = gate ? nullptr : c->latch_stat;      // the gated call has its own rule
+  a.cur_layer = c->cur_layer;
   ASL_CUDA(cudaMemsetAsync(a.scratch, 0, (size_t)segments * SEG_INTS * sizeof(int32_t), st));
   const dim3 grid(tiles, n_heads, c->p.batch);
   topk_digit_kernel<0><<<grid, THREADS, 0, st>>>(a);

@@ -9,7 +9,7 @@ import torch
 from oracle import asl_oracle as O
 from paper_2601_07667_b200 import inputs as I
 
-from asl_check import StatReplay, check_layer, make_path, to_dev
+from asl_check import StatReplay, bits_of, check_layer, make_path, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -380,6 +380,79 @@ def test_device_side_controller_latches_the_selection_and_gates_the_one_shot_top
         want = O.select_tokens(aggs[L][ts:ts + T], wl.budgets[b], wl.seqlens[b], wl.window)
         assert np.array_equal(sel[ko:ko + kept], want)
     path.close()
+
+
+def test_work_of_finished_requests_is_skipped_under_the_latch():
+    """Algorithm 2 ends the method for a request at its selection layer.  With the device-side
+    controller and the layer clock (LayerPath.set_controller) the scorer, the pooling, the per-head
+    top-k and the compaction leave a finished request alone: the outputs of the requests still under
+    observation are bit for bit those of the run that skips nothing, and everything a finished request
+    owns (scores, kept lists, compacted cache, rank rows, record) stays as its selection layer left it."""
+    import dataclasses
+    from paper_2601_07667_b200 import binding as B
+    base = I.workload("C4", seqlens=(3000, 5001, 2177), budgets=(300, 500, 217), layers=7, l_min=1, l_obs=3,
+                      salience_start=0.0, salience_step=0.5)
+    xs = [I.layer_inputs(base, l, seed=11) for l in range(base.layers)]
+    dev = [(to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])) for x in xs]
+
+    def run(wl, mode):
+        """mode 0: report every layer; 1: latch, nothing skipped (no layer clock); 2: latch with skipping"""
+        path = make_path(wl, tail_streams=2)
+        if mode == 1:
+            B.asl_set_controller(path.ctx, B.ASL_CONTROLLER_LATCH)
+        elif mode == 2:
+            path.set_controller(B.ASL_CONTROLLER_LATCH)
+        snaps = []
+        for l in range(wl.layers):
+            path.run_layer(*dev[l], l)
+            torch.cuda.synchronize()
+            snaps.append({"kv": [t.cpu().numpy().copy() for t in path._kv], "agg": [t.cpu().numpy().copy() for t in path._agg],
+                          "cur": path._cur, "idx": path.idx.cpu().numpy().copy(), "k": bits_of(path.k_out).copy(),
+                          "v": bits_of(path.v_out).copy(), "ring": path.rank_ring.cpu().numpy().copy(),
+                          "stat": path.read_stat().copy()})
+        if mode == 2:
+            # a new prompt on the same context: the requests that were left out are scored again (their
+            # publish counters were advanced while they were skipped) and every layer comes out as before
+            path.reset()
+            for l in range(wl.layers):
+                path.run_layer(*dev[l], l)
+                torch.cuda.synchronize()
+                assert np.array_equal(path.idx.cpu().numpy(), snaps[l]["idx"])
+                assert np.array_equal(path.read_stat(), snaps[l]["stat"])
+        assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+        launches = B.asl_launch_count(path.ctx)
+        offs = (path.t_off, path.kept_off)
+        path.close()
+        return snaps, offs, launches
+
+    never = dataclasses.replace(base, tau=0.0)
+    s0, (t_off, kept_off), _ = run(never, 0)
+    rel = np.array([[st["stat"][b]["rel"] for b in range(base.batch)] for st in s0 if st["stat"][0]["evaluated"]])
+    wl = dataclasses.replace(base, tau=float(min(np.median(rel[1:-1]), 0.999)))
+    full, _, _ = run(wl, 1)
+    skip, _, _ = run(wl, 2)
+    sel_layer = [int(full[-1]["stat"][b]["layer_idx"]) if full[-1]["stat"][b]["selected"] else -1 for b in range(wl.batch)]
+    assert any(0 <= L < wl.layers - 2 for L in sel_layer), sel_layer          # somebody finishes with layers to go
+    for l in range(wl.layers):
+        for b in range(wl.batch):
+            T, kept = wl.seqlens[b] - wl.window, wl.kept(b)
+            ts, ko = int(t_off[b]), int(kept_off[b])
+            L = sel_layer[b]
+            seg = lambda sn: (sn["idx"][:, ko:ko + kept], sn["k"][:, ko:ko + kept], sn["v"][:, ko:ko + kept],
+                              sn["ring"][:, ts:ts + T], sn["stat"][b])
+            if L < 0 or l <= L:                                   # still observed at layer l: nothing may differ
+                cur = skip[l]["cur"]
+                assert cur == full[l]["cur"]
+                assert np.array_equal(skip[l]["kv"][cur][:, ts:ts + T], full[l]["kv"][cur][:, ts:ts + T])
+                assert np.array_equal(skip[l]["agg"][cur][ts:ts + T], full[l]["agg"][cur][ts:ts + T])
+                for a_, b_ in zip(seg(skip[l]), seg(full[l])):
+                    assert np.array_equal(a_, b_)
+            else:                                                 # finished: as the selection layer left it
+                for a_, b_ in zip(seg(skip[l]), seg(skip[L])):
+                    assert np.array_equal(a_, b_)
+                for i in range(2):
+                    assert np.array_equal(skip[l]["kv"][i][:, ts:ts + T], skip[L]["kv"][i][:, ts:ts + T])
+                    assert np.array_equal(skip[l]["agg"][i][ts:ts + T], skip[L]["agg"][i][ts:ts + T])
 
 
 def test_layers_replayed_from_a_cuda_graph_match_the_calls():
