@@ -45,6 +45,26 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
     return u32.view(np.float32).astype(np.float64)
 
 
+def widen_fp8_e4m3(codes: np.ndarray) -> np.ndarray:
+    """FP8 E4M3 bit patterns (uint8; the "finite" variant of the OCP 8-bit format: one sign bit, four
+    exponent bits with bias 7, three mantissa bits, no infinities, S.1111.111 = NaN) -> float64, exactly.
+    A quantised K cache stores these codes with one fp32 scale per kv head; the keys the method sees
+    are code value x scale (Algorithm 1 takes K as given)."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(np.float64)
+    normal = np.ldexp(1.0 + m / 8.0, (e - 7).astype(np.int64))
+    subnormal = np.ldexp(m / 8.0, -6)
+    v = sign * np.where(e == 0, subnormal, normal)
+    return np.where((c & 0x7F) == 0x7F, np.nan, v)
+
+
+def dequantised_keys(codes: np.ndarray, k_scale: np.ndarray) -> np.ndarray:
+    """Keys of a quantised cache: codes [n][H_k][d] x one scale per kv head, in float64."""
+    return widen_fp8_e4m3(codes) * np.asarray(k_scale, dtype=np.float64)[None, :, None]
+
+
 # --------------------------------------------------------------------------
 # Algorithm 1: window softmax A and the past-only column sum U
 # --------------------------------------------------------------------------

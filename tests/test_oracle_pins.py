@@ -11,6 +11,7 @@ import pytest
 import torch
 
 from oracle import asl_oracle as O
+from paper_2601_07667_b200 import inputs as I
 
 
 def rng(seed):
@@ -339,3 +340,43 @@ def test_select_tokens_is_the_union_of_best_ranks_and_window():
     order = sorted(range(T), key=lambda j: (-agg[j], j))        # brute force: best k, ties to the lower index
     assert sorted(order[:k]) == sel[:k].tolist()
     assert (O.select_tokens(agg, 10 ** 6, T + w, w) == np.arange(T + w)).all()      # budget >= n keeps everything
+
+
+# ---------------------------------------------------------------- FP8 (E4M3) keys
+def test_fp8_e4m3_decode_literal_values():
+    """Bit patterns whose values follow from the format's definition: 1 sign, 4 exponent bits (bias 7),
+    3 mantissa bits, subnormals at exponent 0, largest finite value 448, S.1111.111 is NaN."""
+    codes = np.array([0x00, 0x80, 0x38, 0xB8, 0x40, 0x3C, 0x7E, 0xFE, 0x01, 0x07, 0x08, 0x30, 0x47], dtype=np.uint8)
+    want = [0.0, -0.0, 1.0, -1.0, 2.0, 1.5, 448.0, -448.0, 2.0 ** -9, 7 * 2.0 ** -9, 2.0 ** -6, 0.5, 3.75]
+    got = O.widen_fp8_e4m3(codes)
+    assert got.tolist() == want
+    assert np.signbit(got[1]) and not np.signbit(got[0])
+    assert np.isnan(O.widen_fp8_e4m3(np.array([0x7F, 0xFF], dtype=np.uint8))).all()
+
+
+def test_fp8_e4m3_decode_agrees_with_the_library_type_on_all_codes():
+    codes = np.arange(256, dtype=np.uint8)
+    lib = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    got = O.widen_fp8_e4m3(codes)
+    assert np.array_equal(np.isnan(got), np.isnan(lib))
+    ok = ~np.isnan(lib)
+    assert np.array_equal(got[ok], lib[ok]) and np.array_equal(np.signbit(got[ok]), np.signbit(lib[ok]))
+    # strictly increasing over the positive codes, symmetric in the sign bit
+    assert (np.diff(got[0:0x7F]) > 0).all() and np.array_equal(got[0x80:0xFF], -got[0x00:0x7F])
+
+
+def test_fp8_key_copy_is_the_nearest_code_and_scales_per_head():
+    """The input helper's codes: no other code is nearer to k/scale, the head's largest key maps to 448."""
+    g = np.random.default_rng(5)
+    k = (g.standard_normal((40, 3, 16)) * np.array([0.3, 1.0, 20.0])[None, :, None]).astype(np.float32)
+    bits = I.f32_to_bf16_bits(k)
+    codes, scale = I.keys_to_fp8(bits)
+    assert codes.dtype == np.uint8 and codes.shape == k.shape and scale.shape == (3,)
+    exact = I.bf16_bits_to_f64(bits) / scale.astype(np.float64)[None, :, None]
+    table = O.widen_fp8_e4m3(np.arange(0x7F, dtype=np.uint8))             # all non-negative finite values
+    err = np.abs(np.abs(O.widen_fp8_e4m3(codes)) - np.abs(exact))
+    best = np.abs(np.abs(exact)[..., None] - table).min(axis=-1)
+    assert (err <= best * (1 + 1e-6) + 1e-12).all()
+    assert (np.abs(O.widen_fp8_e4m3(codes)).max(axis=(0, 2)) == 448.0).all()
+    deq = O.dequantised_keys(codes, scale)
+    assert np.abs(deq - I.bf16_bits_to_f64(bits)).max() <= 20.0 * 5 / 16      # 3 mantissa bits: relative step 1/8
