@@ -62,7 +62,7 @@ def peaks():
     return p
 
 
-def algorithmic_work(wl):
+def algorithmic_work(wl, fp8_keys=False):
     """Algorithmic bytes and flops of one layer's pass: K read once, Q once, only
     kept K/V rows gathered (read + write), score vectors written and re-read by
     the pooling, ranking and selection stages, one QK^T."""
@@ -70,9 +70,9 @@ def algorithmic_work(wl):
     n_tot = wl.total_tokens
     T_tot = n_tot - wl.batch * w
     kept = sum(wl.kept(b) for b in range(wl.batch))
-    k_bytes = n_tot * Hk * d * 2
+    k_bytes = n_tot * Hk * d * (1 if fp8_keys else 2)
     q_bytes = wl.batch * w * Hq * d * 2
-    gather = 4 * kept * Hk * d * 2
+    gather = (2 if fp8_keys else 4) * kept * Hk * d + 4 * kept * Hk * d      # K rows (1 or 2 bytes/element) + V rows, read + write
     score = 3 * (Hk + 1) * T_tot * 4 + kept * Hk * 4
     flops = 2.0 * w * d * n_tot * Hq
     return {"bytes": k_bytes + q_bytes + gather + score, "k_bytes": k_bytes, "flops": flops,
@@ -301,21 +301,31 @@ def run_ours(args):
     wl = make_workload(args)
     if args.score_ctas < 0:
         args.score_ctas = max(1, torch.cuda.get_device_properties(local).multi_processor_count + args.score_ctas)
-    work = algorithmic_work(wl)
+    fp8 = args.k_dtype == "fp8"
+    work = algorithmic_work(wl, fp8)
     pk = peaks()
 
     # resident inputs: a few layers' tensors, rotated (each rank draws its own seed: independent requests)
     n_sets = args.layer_sets
     host_sets = [I.layer_inputs(wl, l, rank_seed(args.seed, rank)) for l in range(n_sets)]
-    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    k_scale = None
+    if fp8:
+        # a quantised K cache: one scale per kv head for the whole run (the scales belong to the plan)
+        amax = np.max([np.abs(I.bf16_bits_to_f32(x["k"])).max(axis=(0, 2)) for x in host_sets], axis=0)
+        k_scale = (amax / 448.0).astype(np.float32)
+        for x in host_sets:
+            x["k"] = I.keys_to_fp8(x["k"], k_scale)[0]
+    pin = lambda a: torch.from_numpy(a if a.dtype == np.uint8 else a.view(np.int16)).pin_memory()
     host_pinned = [{k: pin(x[k]) for k in ("q_obs", "k", "v")} for x in host_sets]
-    dev_sets = [{k: t.cuda(non_blocking=True).view(torch.bfloat16) for k, t in hp.items()} for hp in host_pinned]
+    as_dev = lambda t: t.cuda(non_blocking=True) if t.dtype == torch.uint8 else t.cuda(non_blocking=True).view(torch.bfloat16)
+    dev_sets = [{k: as_dev(t) for k, t in hp.items()} for hp in host_pinned]
     torch.cuda.synchronize()
 
     path = B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
                        pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
                        l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=args.score_ctas,
-                       tail_streams=args.tail_streams)
+                       tail_streams=args.tail_streams, k_dtype=B.ASL_K_FP8_E4M3 if fp8 else B.ASL_K_BF16,
+                       k_scale=None if k_scale is None else [float(s) for s in k_scale])
 
     def barrier():
         if world > 1:
@@ -445,15 +455,14 @@ def run_ours(args):
     e2e_steps = max(2, min(args.steps, args.e2e_steps))
     q_d, k_d, v_d = (torch.empty_like(dev_sets[0][k]) for k in ("q_obs", "k", "v"))
     idx_h = torch.empty(path.idx.shape, dtype=torch.int32).pin_memory()
-    ko_h = torch.empty(path.k_out.shape, dtype=torch.bfloat16).pin_memory()
+    ko_h = torch.empty(path.k_out.shape, dtype=path.k_out.dtype).pin_memory()
     vo_h = torch.empty(path.v_out.shape, dtype=torch.bfloat16).pin_memory()
     st_h = torch.empty(path.stat.shape, dtype=torch.uint8).pin_memory()
 
     def e2e_step(i):
         hp = host_pinned[i % n_sets]
-        q_d.view(torch.int16).copy_(hp["q_obs"], non_blocking=True)
-        k_d.view(torch.int16).copy_(hp["k"], non_blocking=True)
-        v_d.view(torch.int16).copy_(hp["v"], non_blocking=True)
+        for dst, key in ((q_d, "q_obs"), (k_d, "k"), (v_d, "v")):
+            (dst if dst.dtype == torch.uint8 else dst.view(torch.int16)).copy_(hp[key], non_blocking=True)
         path.run_layer(q_d, k_d, v_d, i)
         path.join()                     # top-k, compaction and the statistic run on side streams
         idx_h.copy_(path.idx, non_blocking=True)
@@ -472,11 +481,11 @@ def run_ours(args):
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / e2e_steps
     # the leg checks what it timed: the host copies are the device results of the last step
-    if not (torch.equal(idx_h, path.idx.cpu()) and torch.equal(ko_h.view(torch.int16), path.k_out.cpu().view(torch.int16))
+    if not (torch.equal(idx_h, path.idx.cpu()) and torch.equal(ko_h.view(torch.uint8), path.k_out.cpu().view(torch.uint8))
             and torch.equal(st_h, path.stat.cpu())):
         raise SystemExit("end-to-end leg: host copies differ from the device results")
-    h2d = sum(host_pinned[0][k].numel() * 2 for k in ("q_obs", "k", "v"))
-    d2h = idx_h.numel() * 4 + ko_h.numel() * 2 + vo_h.numel() * 2 + st_h.numel()
+    h2d = sum(host_pinned[0][k].numel() * host_pinned[0][k].element_size() for k in ("q_obs", "k", "v"))
+    d2h = idx_h.numel() * 4 + ko_h.numel() * ko_h.element_size() + vo_h.numel() * 2 + st_h.numel()
 
     if rank != 0:
         if world > 1:
@@ -485,7 +494,7 @@ def run_ours(args):
 
     # ---- roofline of the whole step and of the scorer ----
     hbm = pk["hbm_gbs"]
-    tf = pk["bf16_tflops"]
+    tf = pk["bf16_tflops"] * (2.0 if fp8 else 1.0)      # 8-bit operands: the measured bf16 peak times the nominal fp8/bf16 ratio
     t_hbm = work["bytes"] / (hbm * 1e9)
     t_mma = work["flops"] / (tf * 1e12)
     bound = "hbm" if t_hbm >= t_mma else "tensor"
@@ -495,14 +504,14 @@ def run_ours(args):
     else:
         achieved = work["flops"] / (score_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": tf, "unit": "TFLOP/s", "frac": achieved / tf}
-    default_shape = not args.seqlens and not args.budgets and not args.heads
+    default_shape = not args.seqlens and not args.budgets and not args.heads and not fp8
     roof.update({"traffic": scorer_traffic_bytes(wl.name) if default_shape else None, "kernel": "score_tc_kernel (asl_score_columns: both softmax passes, one persistent launch)", "kernel_ms": score_ms,
                  "peak_source": pk["source"], "step_roofline_us": max(t_hbm, t_mma) * 1e6,
                  "step_frac": max(t_hbm, t_mma) / (ms_step * 1e-3)})
 
     # ---- the oracle on the host cores, bounded sample ----
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not fp8:
         v, dt = time_oracle(wl, host_sets, 2, 1, 1)
         cpu = {"value": v, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                "sample": f"2 layers, kv head 0 with its {wl.group} query heads (1/{wl.n_kv_heads} of scoring, top-k and "
@@ -513,7 +522,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "seqlens": list(wl.seqlens), "window": wl.window,
                        "budgets": list(wl.budgets), "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv", "d": wl.head_dim,
-                       "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"],
+                       "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"], "k_dtype": args.k_dtype,
                        "l2": (f"inputs larger than L2: {n_sets} resident layer sets rotated, K = "
                               f"{work['k_bytes'] / 1e6:.0f} MB per layer") if work["k_bytes"] * n_sets > 126e6 else
                              (f"small workload: {n_sets} layer sets of {work['k_bytes'] / 1e6:.1f} MB K stay in L2 "
@@ -555,6 +564,8 @@ def main():
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")
     ap.add_argument("--heads", type=str, default=None, help="query,kv head counts replacing the workload's (e.g. 28,4)")
+    ap.add_argument("--k-dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: K as E4M3 codes with one scale per kv head (a quantised K cache); the headline workload is bf16")
     ap.add_argument("--dry-run", action="store_true",
                     help="ranks only rendezvous and reduce a fixed time (checks the multi-rank launch; runs no kernel)")
     args = ap.parse_args()

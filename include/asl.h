@@ -68,6 +68,7 @@ typedef enum {
 } asl_status;
 
 enum { ASL_POOL_AVG = 0, ASL_POOL_MAX = 1 };
+enum { ASL_K_BF16 = 0, ASL_K_FP8_E4M3 = 1 };   /* element type of K */
 
 /* Problem statement of Algorithm 1 (W, S, KV_budget) and Algorithm 2
  * (L_min, L_obs, tau).  Host arrays are copied by asl_plan. */
@@ -90,6 +91,18 @@ typedef struct {
   int64_t q_stride[3];    /* q_obs element strides: request, head, row                */
   int64_t k_stride[2];    /* K element strides: token, head                           */
   int64_t v_stride[2];    /* V element strides: token, head                           */
+  int32_t k_dtype;        /* ASL_K_BF16, or ASL_K_FP8_E4M3: a quantised K cache.  K then  */
+                          /* holds 8-bit E4M3 codes (finite variant: no infinities) and   */
+                          /* the key the method sees is code x k_scale[kv head]; k_stride */
+                          /* counts 1-byte elements, rows still start on 16-byte          */
+                          /* boundaries; asl_compact_kv copies the codes (k_out is        */
+                          /* [H_k][sum_kept][d] bytes), V stays bf16.  The queries stay   */
+                          /* bf16: the scorer splits each into two E4M3 terms (exact for  */
+                          /* 1/64 <= |q| <= 28, else to 2^-13 / saturated) and runs the   */
+                          /* contraction on the 8-bit tensor-core path.  Shapes the       */
+                          /* tensor-core scorer does not take are ASL_ERR_UNSUPPORTED.    */
+  int32_t reserved0;
+  const float* k_scale;   /* host [H_k], finite and > 0; read only for ASL_K_FP8_E4M3     */
 } asl_params;
 
 /* Result of Algorithm 2 for one request; lives in device memory, [B] of them,

@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libasl_b200.so")
 
 ASL_POOL_AVG, ASL_POOL_MAX = 0, 1
+ASL_K_BF16, ASL_K_FP8_E4M3 = 0, 1
 ASL_OK, ASL_ERR_INVALID, ASL_ERR_UNSUPPORTED, ASL_ERR_WORKSPACE = 0, -1, -2, -3
 ASL_ERR_CUDA, ASL_ERR_TIMEOUT, ASL_ERR_ARCH = -4, -5, -6
 
@@ -31,7 +32,8 @@ class AslParams(C.Structure):
                 ("batch", C.c_int32), ("l_min", C.c_int32), ("l_obs", C.c_int32), ("score_ctas", C.c_int32),
                 ("tau", C.c_double),
                 ("cu_seqlens", C.POINTER(C.c_int32)), ("budgets", C.POINTER(C.c_int32)),
-                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 2), ("v_stride", C.c_int64 * 2)]
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 2), ("v_stride", C.c_int64 * 2),
+                ("k_dtype", C.c_int32), ("reserved0", C.c_int32), ("k_scale", C.POINTER(C.c_float))]
 
 
 class AslStat(C.Structure):
@@ -136,12 +138,15 @@ def asl_destroy(ctx: int) -> None:
 def asl_plan(ctx: int, *, n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, pool_kernel: int,
              pool_mode: int, cu_seqlens: Sequence[int], budgets: Sequence[int], l_min: int, l_obs: int,
              tau: float, q_stride: Sequence[int], k_stride: Sequence[int], v_stride: Sequence[int],
-             score_ctas: int = 0) -> int:
+             score_ctas: int = 0, k_dtype: int = ASL_K_BF16, k_scale: Optional[Sequence[float]] = None) -> int:
     cu = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
     bu = (C.c_int32 * len(budgets))(*[int(x) for x in budgets])
+    ks = (C.c_float * len(k_scale))(*[float(x) for x in k_scale]) if k_scale is not None else None
     p = AslParams(n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, len(budgets), l_min, l_obs, int(score_ctas),
                   float(tau), cu, bu, (C.c_int64 * 3)(*q_stride), (C.c_int64 * 2)(*k_stride),
-                  (C.c_int64 * 2)(*v_stride))
+                  (C.c_int64 * 2)(*v_stride), int(k_dtype), 0, ks)
+    if k_scale is not None and len(k_scale) != n_kv_heads:
+        raise AslError(ASL_ERR_INVALID, "asl_plan")
     if len(cu_seqlens) != len(budgets) + 1:
         raise AslError(ASL_ERR_INVALID, "asl_plan")
     size = C.c_size_t(0)
@@ -257,7 +262,7 @@ class LayerPath:
 
     def __init__(self, *, n_q_heads, n_kv_heads, head_dim, window, pool_kernel, pool_mode, seqlens, budgets,
                  l_min, l_obs, tau, device: int = 0, q_stride=None, k_stride=None, v_stride=None,
-                 score_ctas: int = 0, tail_streams: int = 1):
+                 score_ctas: int = 0, tail_streams: int = 1, k_dtype: int = ASL_K_BF16, k_scale=None):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda", device)
@@ -274,7 +279,8 @@ class LayerPath:
         self.ws_bytes = asl_plan(self.ctx, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
                                  window=window, pool_kernel=pool_kernel, pool_mode=pool_mode, cu_seqlens=cu,
                                  budgets=budgets, l_min=l_min, l_obs=l_obs, tau=tau, q_stride=q_stride,
-                                 k_stride=k_stride, v_stride=v_stride, score_ctas=score_ctas)
+                                 k_stride=k_stride, v_stride=v_stride, score_ctas=score_ctas, k_dtype=k_dtype,
+                                 k_scale=k_scale)
         self.sum_tokens, self.sum_T, self.sum_kept = asl_plan_sizes(self.ctx)
         self.kept = [min(int(bg), n) for bg, n in zip(budgets, self.seqlens)]
         self.t_off = np.concatenate([[0], np.cumsum([n - window for n in self.seqlens])]).astype(np.int64)
@@ -286,7 +292,8 @@ class LayerPath:
         self._agg_free = [None, None]       # event after the side-stream work that last read the buffers
         self._cur = 0
         self.idx = torch.empty((n_kv_heads, self.sum_kept), dtype=torch.int32, device=dev)
-        self.k_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
+        self.k_out = torch.empty((n_kv_heads, self.sum_kept, head_dim),
+                                 dtype=torch.uint8 if k_dtype == ASL_K_FP8_E4M3 else torch.bfloat16, device=dev)
         self.v_out = torch.empty((n_kv_heads, self.sum_kept, head_dim), dtype=torch.bfloat16, device=dev)
         self.rank_ring = torch.zeros((l_obs, self.sum_T), dtype=torch.int32, device=dev)
         self.stat = torch.zeros((self.batch, C.sizeof(AslStat)), dtype=torch.uint8, device=dev)

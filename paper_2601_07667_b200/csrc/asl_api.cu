@@ -66,6 +66,14 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   if (p->l_obs < 2 || p->l_min < 0 || p->score_ctas < 0) return ASL_ERR_INVALID;
   if (p->head_dim < 8 || p->head_dim % 8) return ASL_ERR_INVALID;
   if (p->head_dim != 128) return ASL_ERR_UNSUPPORTED;
+  if (p->k_dtype != ASL_K_BF16 && p->k_dtype != ASL_K_FP8_E4M3) return ASL_ERR_INVALID;
+  const bool fp8 = p->k_dtype == ASL_K_FP8_E4M3;
+  if (fp8) {
+    if (!p->k_scale) return ASL_ERR_INVALID;
+    for (int h = 0; h < p->n_kv_heads; ++h)
+      if (!(p->k_scale[h] > 0.0f) || !(p->k_scale[h] < INFINITY)) return ASL_ERR_INVALID;
+    if (p->k_stride[0] % 16 || p->k_stride[1] % 16) return ASL_ERR_INVALID;     // 16-byte rows of 1-byte elements
+  }
   // rows must start on 16-byte boundaries: every stride a multiple of 8 elements
   const int64_t strides[] = {p->q_stride[0], p->q_stride[1], p->q_stride[2], p->k_stride[0],
                              p->k_stride[1], p->v_stride[0], p->v_stride[1]};
@@ -120,6 +128,10 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   c->budgets.assign(p->budgets, p->budgets + p->batch);
   c->p.cu_seqlens = c->cu.data();
   c->p.budgets = c->budgets.data();
+  c->k_scale.clear();
+  if (fp8) c->k_scale.assign(p->k_scale, p->k_scale + p->n_kv_heads);
+  c->p.k_scale = fp8 ? c->k_scale.data() : nullptr;
+  c->k_elem_bytes = fp8 ? 1 : 2;
   c->req = req;
   c->sum_tokens = p->cu_seqlens[p->batch];
   c->sum_T = sum_T;
@@ -132,6 +144,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   cudaSetDevice(c->device);
   const bool tc = asl_tc_plan(c);
   cudaSetDevice(prev);
+  if (fp8 && !tc) { free_plan(c); return ASL_ERR_UNSUPPORTED; }     // only the tensor-core scorer reads 8-bit keys
   const int G = p->n_q_heads / p->n_kv_heads;
   // the tensor-core scorer writes two partial column sums per chunk (one per half of the chunk's rows);
   // under max pooling they belong to different query heads unless a chunk is a single head
@@ -147,6 +160,8 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   w.score_offsets = off;  off = asl_align256(off + (size_t)p->batch * p->n_kv_heads * rows_padded * sizeof(float));
   const size_t u_rows = (size_t)p->n_kv_heads * c->u_rows_per_kv;
   for (int i = 0; i < 2; ++i) { w.score_u[i] = off; off = asl_align256(off + u_rows * (size_t)sum_T * sizeof(float)); }
+  w.score_q8 = off;
+  if (fp8) off = asl_align256(off + (size_t)2 * p->batch * p->n_q_heads * p->window * p->head_dim);
   w.score_end = off;
   for (int i = 0; i < 2; ++i) { w.rank_keys[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }
   for (int i = 0; i < 2; ++i) { w.rank_idx[i] = off; off = asl_align256(off + (size_t)sum_T * 4); }

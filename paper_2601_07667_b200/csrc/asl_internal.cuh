@@ -25,6 +25,7 @@ struct AslWorkspace {
   size_t score_partials;   // pass-1 partial row statistics
   size_t score_offsets;    // per-row log2 normalisers
   size_t score_u[2];       // un-pooled column sums, two slots
+  size_t score_q8;         // fp8 K: the window queries as two E4M3 terms [2][B][H_q][W][d] bytes
   size_t score_end;
   size_t rank_keys[2];     // ping-pong sort keys
   size_t rank_idx[2];      // ping-pong sort payload
@@ -45,6 +46,8 @@ struct asl_ctx {
   uint32_t* d_skip = nullptr;         // device [8]: bit b set = request b finished before cur_layer (scorer's snapshot)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
+  std::vector<float> k_scale;         // per kv head (fp8 K), else empty
+  int k_elem_bytes = 2;               // bytes per K element
   std::vector<AslReq> req;
   int64_t sum_tokens = 0, sum_T = 0, sum_kept = 0;
   int32_t max_n = 0, max_T = 0, max_kept = 0;

@@ -1,29 +1,32 @@
 // K/V compaction (Algorithm 1 (K[I], V[I])): out[h][r][:] = x[tok_off + idx[h][r]][h][:].
-// 16 threads move one 256-byte row as 16-byte vectors; K and V in one launch.
+// 16 threads move one row (256 bytes of bf16, 128 bytes of FP8 codes) as 16-byte vectors; K and V in one launch.
 #include "asl_internal.cuh"
 
 namespace {
 
-__global__ void __launch_bounds__(256) compact_kv_kernel(const uint16_t* __restrict__ k, const uint16_t* __restrict__ v,
+__global__ void __launch_bounds__(256) compact_kv_kernel(const uint8_t* __restrict__ k, const uint8_t* __restrict__ v,
                                                          const int32_t* __restrict__ idx, const AslReq* __restrict__ req,
                                                          int64_t ks_t, int64_t ks_h, int64_t vs_t, int64_t vs_h,
-                                                         int64_t sum_kept, int vec_per_row, const asl_stat* __restrict__ latch,
-                                                         int cur_layer, uint16_t* __restrict__ k_out,
-                                                         uint16_t* __restrict__ v_out) {
+                                                         int64_t sum_kept, int k_vec, int v_vec, const asl_stat* __restrict__ latch,
+                                                         int cur_layer, uint8_t* __restrict__ k_out,
+                                                         uint8_t* __restrict__ v_out) {
+  // strides in bytes; a row is k_vec (v_vec) 16-byte vectors; 16 threads per kept row
   const int b = blockIdx.z, h = blockIdx.y;
   if (latch && asl_finished(latch + b, cur_layer)) return;       // finished request: its compacted cache is final
   const AslReq rq = req[b];
-  const int rows_per_block = blockDim.x / vec_per_row;
-  const int r = blockIdx.x * rows_per_block + threadIdx.x / vec_per_row;
-  const int c = threadIdx.x % vec_per_row;
+  const int r = blockIdx.x * (blockDim.x / 16) + threadIdx.x / 16;
+  const int c = threadIdx.x % 16;
   if (r >= rq.kept) return;
   const int64_t orow = (int64_t)h * sum_kept + rq.kept_off + r;
   const int64_t tok = (int64_t)rq.tok_off + idx[orow];
-  const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * ks_t + (int64_t)h * ks_h + c * 8);
-  const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * vs_t + (int64_t)h * vs_h + c * 8);
-  const int64_t o = orow * (vec_per_row * 8) + c * 8;
-  *reinterpret_cast<uint4*>(k_out + o) = kv;
-  *reinterpret_cast<uint4*>(v_out + o) = vv;
+  if (c < k_vec) {
+    const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * ks_t + (int64_t)h * ks_h + c * 16);
+    *reinterpret_cast<uint4*>(k_out + (orow * k_vec + c) * 16) = kv;
+  }
+  if (c < v_vec) {
+    const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * vs_t + (int64_t)h * vs_h + c * 16);
+    *reinterpret_cast<uint4*>(v_out + (orow * v_vec + c) * 16) = vv;
+  }
 }
 
 // Row gather of one tensor with rows of `row_bytes` (a multiple of 16): out[kept_off_b + r] = x[tok_off_b + idx[r]].
@@ -55,13 +58,13 @@ asl_status asl_launch_compact_rows(asl_ctx* c, const void* x, const int32_t* idx
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st) {
   const asl_params& p = c->p;
-  const int vec = p.head_dim / 8;                 // 16-byte vectors per row
-  const int rows_per_block = 256 / vec;
-  dim3 grid((c->max_kept + rows_per_block - 1) / rows_per_block, p.n_kv_heads, p.batch);
-  compact_kv_kernel<<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), idx, c->d_req,
-                                          p.k_stride[0], p.k_stride[1], p.v_stride[0], p.v_stride[1], c->sum_kept, vec,
-                                          c->latch_stat, c->cur_layer,
-                                          static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out));
+  const int kb = c->k_elem_bytes;                          // K elements are 2 bytes (bf16) or 1 (FP8 codes), V is bf16
+  const int k_vec = p.head_dim * kb / 16, v_vec = p.head_dim * 2 / 16;
+  dim3 grid((c->max_kept + 15) / 16, p.n_kv_heads, p.batch);
+  compact_kv_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t*>(k), static_cast<const uint8_t*>(v), idx, c->d_req,
+                                          p.k_stride[0] * kb, p.k_stride[1] * kb, p.v_stride[0] * 2, p.v_stride[1] * 2,
+                                          c->sum_kept, k_vec, v_vec, c->latch_stat, c->cur_layer,
+                                          static_cast<uint8_t*>(k_out), static_cast<uint8_t*>(v_out));
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

@@ -36,6 +36,7 @@
 // the epilogue keeps walking its barrier sequence without waiting or computing,
 // in-flight copies are waited for with the same bound and tensor memory is freed.
 #include <cuda.h>
+#include <cuda_fp8.h>
 
 #include "asl_internal.cuh"
 
@@ -159,6 +160,15 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(
+          dst),
+      "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -171,6 +181,15 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+// the same with 8-bit operands (E4M3 x E4M3 -> fp32), 32 channels per instruction
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum)
       : "memory");
 }
@@ -292,6 +311,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
+// kind::f8f6f4, A = B = E4M3 (format code 0), D = fp32, both operands K-major
+__device__ __forceinline__ uint32_t instr_desc_f8(int M, int N) {
+  return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
 
 struct TcArgs {
   const TcPhase* phases;
@@ -338,7 +361,10 @@ struct ItemWalk {
   __device__ __forceinline__ void next() { g += (int)gridDim.x; }
 };
 
-template <bool PER_Q>
+// FP8: K tiles hold E4M3 codes (one 128-byte row per key: a tile is one 16 KB box), the query chunk holds
+// the two E4M3 terms of every query (term t in the t-th 32 KB block of the chunk's buffer, where bf16
+// queries keep their t-th 64-channel block), and a tile takes 2 terms x 4 k-steps of 32 channels.
+template <bool PER_Q, bool FP8>
 __global__ void __launch_bounds__(THREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -418,8 +444,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const int head = p.h * a.G + r0 / a.W, t0 = r0 % a.W;
           const uint32_t dst = sbase + SM_Q + (uint32_t)b * Q_BUF_BYTES;
           mbar_expect_tx(bar(BAR_QFULL + b), 2u * 128u * (uint32_t)NC);
-          tma_load_4d(dst, &tm_q, bar(BAR_QFULL + b), 0, t0, head, p.b);
-          tma_load_4d(dst + Q_BLOCK_BYTES, &tm_q, bar(BAR_QFULL + b), 64, t0, head, p.b);
+          if (FP8) {
+            tma_load_5d(dst, &tm_q, bar(BAR_QFULL + b), 0, t0, head, p.b, 0);
+            tma_load_5d(dst + Q_BLOCK_BYTES, &tm_q, bar(BAR_QFULL + b), 0, t0, head, p.b, 1);
+          } else {
+            tma_load_4d(dst, &tm_q, bar(BAR_QFULL + b), 0, t0, head, p.b);
+            tma_load_4d(dst + Q_BLOCK_BYTES, &tm_q, bar(BAR_QFULL + b), 64, t0, head, p.b);
+          }
           loaded_seg[b] = p.seg;
         }
         q_issued = l;
@@ -449,12 +480,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         const int s = item % NSTAGE;
         if (!mbar_wait(bar(BAR_EMPTY + s), ((item / NSTAGE) & 1) ^ 1, s_abort, 12, true)) { ok = false; break; }
-        mbar_expect_tx(bar(BAR_FULL + s), STAGE_BYTES);
+        mbar_expect_tx(bar(BAR_FULL + s), FP8 ? HALF_BYTES : STAGE_BYTES);
         const uint32_t dst = sbase + SM_K + s * STAGE_BYTES;
         const int tok = tok_off + (w.g - p.g0) * KT;
         const uint64_t pol = p.pass == 1 ? pol_keep : pol_stream;
         tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok, pol);
-        tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok, pol);
+        if (!FP8) tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok, pol);
         ++item;
       }
       if (!ok) {
@@ -474,7 +505,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       ItemWalk w(a);
       int item = 0, lp = -1, cur_ph = -1;
       bool ok = true;
-      const uint32_t idesc1 = instr_desc(128, KT), idesc2 = instr_desc(KT, NC);
+      const uint32_t idesc1 = FP8 ? instr_desc_f8(128, KT) : instr_desc(128, KT);
+      const uint32_t idesc2 = FP8 ? instr_desc_f8(KT, NC) : instr_desc(KT, NC);
+      // byte offset of k-step ks inside a K tile: bf16 tiles are two 64-channel blocks, 8-bit tiles one block
+      auto k_off = [](int ks) { return (uint32_t)(FP8 ? (ks & 3) * 32 : (ks >> 2) * HALF_BYTES + (ks & 3) * 32); };
       const int nhalf = (NC > 128) ? 2 : 1;
       uint32_t qbase = 0;
       for (; ok && w.valid(); w.next()) {
@@ -495,17 +529,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (p.pass == 2) {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t ad = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
+            const uint64_t ad = smem_desc(kbase + k_off(ks));
             const uint64_t bd = smem_desc(qbase + (ks >> 2) * Q_BLOCK_BYTES + (ks & 3) * 32);
-            tc_mma(d0, ad, bd, idesc2, ks > 0);
+            if (FP8) tc_mma_f8(d0, ad, bd, idesc2, ks > 0);
+            else     tc_mma(d0, ad, bd, idesc2, ks > 0);
           }
         } else {
           for (int hf = 0; hf < nhalf; ++hf) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const uint64_t ad = smem_desc(qbase + (ks >> 2) * Q_BLOCK_BYTES + hf * (128 * 128) + (ks & 3) * 32);
-              const uint64_t bd = smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32);
-              tc_mma(d0 + (uint32_t)(hf * 128), ad, bd, idesc1, ks > 0);
+              const uint64_t bd = smem_desc(kbase + k_off(ks));
+              if (FP8) tc_mma_f8(d0 + (uint32_t)(hf * 128), ad, bd, idesc1, ks > 0);
+              else     tc_mma(d0 + (uint32_t)(hf * 128), ad, bd, idesc1, ks > 0);
             }
           }
         }
@@ -582,8 +618,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int lt = quarter * 32 + lane;                        // TMEM lane of this thread, 0..127
     const int st = (e & 7) * 32 + lane;                        // thread of the set, 0..255
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 256);
-    const float scale = a.scale_log2;
-    const f32x2 scale2 = pk(scale, scale);
+    float scale = a.scale_log2;             // log2(e)/sqrt(d) times the phase's accumulator factor (FP8 keys: per kv head)
+    f32x2 scale2 = pk(scale, scale);
     float* negoff = s_negoff + set * 256;
     const int nhalf = (NC > 128) ? 2 : 1;
     ItemWalk w(a);
@@ -599,6 +635,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (skipped(p.b)) continue;
       if (w.ph != cur_ph) {
         cur_ph = w.ph;
+        if (FP8) {
+          scale = a.scale_log2 * p.kscale;
+          scale2 = pk(scale, scale);
+        }
         if (p.pass == 1) {
           mref = -INFINITY;
           l = 0.f;
@@ -805,6 +845,27 @@ __global__ void bounded_wait_selftest_kernel(int which, unsigned long long limit
   if (threadIdx.x == 0 && !ok && *abort_flag) atomicCAS(err, 0, *abort_flag);
 }
 
+// FP8 keys: the bf16 window queries, scaled by Q8_SCALE, as two E4M3 terms hi + lo (hi = nearest code,
+// lo = nearest code of the remainder; together exact whenever the remainder's bits fit the format, i.e.
+// for 1/64 <= |q| <= 28): out[t][b][head][row][c], dense.
+constexpr float Q8_SCALE = 16.0f;
+__global__ void __launch_bounds__(256) split_queries_e4m3_kernel(const __nv_bfloat16* __restrict__ q, int64_t qs_b, int64_t qs_h,
+                                                                 int64_t qs_r, int Hq, int W, int64_t total,
+                                                                 uint8_t* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i & 127);
+  const int64_t r = i >> 7;
+  const int row = (int)(r % W), head = (int)((r / W) % Hq);
+  const int64_t b = r / ((int64_t)W * Hq);
+  const float x = __bfloat162float(q[b * qs_b + head * qs_h + row * qs_r + c]) * Q8_SCALE;
+  const __nv_fp8_storage_t hi = __nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
+  const float xh = __half2float(__half(__nv_cvt_fp8_to_halfraw(hi, __NV_E4M3)));
+  const __nv_fp8_storage_t lo = __nv_cvt_float_to_fp8(x - xh, __NV_SATFINITE, __NV_E4M3);
+  out[i] = hi;
+  out[total + i] = lo;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -821,12 +882,12 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-bool make_map(CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-              const cuuint32_t* box) {
+bool make_map(CUtensorMap* tm, CUtensorMapDataType dtype, const void* base, int rank, const cuuint64_t* dims,
+              const cuuint64_t* strides_bytes, const cuuint32_t* box) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides_bytes, box, estr,
+  return fn(tm, dtype, rank, const_cast<void*>(base), dims, strides_bytes, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -875,7 +936,7 @@ bool asl_tc_plan(asl_ctx* c) {
   // row denominators; K of a whole group has to stay in L2 between the passes (72 MB of the 126 MB).
   int group = 0;
   {
-    const double seg_bytes = (double)c->sum_tokens * p.k_stride[0] * 2.0 / p.n_kv_heads / (double)p.batch;   // one kv head of an average request
+    const double seg_bytes = (double)c->sum_tokens * p.k_stride[0] * c->k_elem_bytes / p.n_kv_heads / (double)p.batch;   // one kv head of an average request
     group = (int)(72.0e6 / (seg_bytes > 1.0 ? seg_bytes : 1.0));
     group = group < 1 ? 1 : (group > 16 ? 16 : group);
   }
@@ -889,6 +950,7 @@ bool asl_tc_plan(asl_ctx* c) {
     ph.ncontrib = segs[s].tiles1 < tp.grid ? segs[s].tiles1 : tp.grid;    // CTAs with a tile in pass 1
     ph.T = c->req[ph.b].T; ph.t_off = c->req[ph.b].t_off; ph.tok_off = c->req[ph.b].tok_off;
     ph.rows = R - ph.chunk * NC < NC ? R - ph.chunk * NC : NC;
+    ph.kscale = p.k_dtype == ASL_K_FP8_E4M3 ? c->k_scale[ph.h] / Q8_SCALE : 1.0f;
     g += ph.ntiles;
     tp.phases.push_back(ph);
   };
@@ -915,8 +977,10 @@ bool asl_tc_plan(asl_ctx* c) {
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases, tp.phases.data(), tp.phases.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(tp.d_sync, 0, sync_bytes);
   if (e != cudaSuccess) { asl_tc_free(c); return false; }
-  cudaFuncSetAttribute(score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  cudaFuncSetAttribute(score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaFuncSetAttribute(score_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaFuncSetAttribute(score_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaFuncSetAttribute(score_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaFuncSetAttribute(score_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (cudaGetLastError() != cudaSuccess) { asl_tc_free(c); return false; }
   tp.enabled = encode_fn() != nullptr;
   return tp.enabled;
@@ -958,19 +1022,33 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   const asl_params& p = c->p;
   AslTcPlan& tp = c->tc;
   const int W = p.window, G = p.n_q_heads / p.n_kv_heads, NC = tp.NC;
+  const bool fp8 = p.k_dtype == ASL_K_FP8_E4M3;
   CUtensorMap tm_q, tm_k;
-  {
+  const cuuint32_t bw = (cuuint32_t)(W < NC ? W : NC);
+  if (fp8) {
+    // the queries as two E4M3 terms in the workspace, then 8-bit maps: rows of 128 one-byte channels
+    uint8_t* q8 = reinterpret_cast<uint8_t*>(ws + c->ws.score_q8);
+    const int64_t total = (int64_t)p.batch * p.n_q_heads * W * 128;
+    split_queries_e4m3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(q), p.q_stride[0], p.q_stride[1], p.q_stride[2], p.n_q_heads, W, total, q8);
+    c->launches += 1;
+    const cuuint64_t qdims[5] = {128, (cuuint64_t)W, (cuuint64_t)p.n_q_heads, (cuuint64_t)p.batch, 2};
+    const cuuint64_t qstr[4] = {128, (cuuint64_t)W * 128, (cuuint64_t)p.n_q_heads * W * 128, (cuuint64_t)total};
+    const cuuint32_t qbox[5] = {128, bw, (cuuint32_t)NC / bw, 1, 1};
+    if (!make_map(&tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, q8, 5, qdims, qstr, qbox)) return ASL_ERR_CUDA;
+    const cuuint64_t kdims[3] = {128, (cuuint64_t)p.n_kv_heads, (cuuint64_t)c->sum_tokens};
+    const cuuint64_t kstr[2] = {(cuuint64_t)p.k_stride[1], (cuuint64_t)p.k_stride[0]};
+    const cuuint32_t kbox[3] = {128, 1, (cuuint32_t)KT};
+    if (!make_map(&tm_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, k, 3, kdims, kstr, kbox)) return ASL_ERR_CUDA;
+  } else {
     const cuuint64_t dims[4] = {128, (cuuint64_t)W, (cuuint64_t)p.n_q_heads, (cuuint64_t)p.batch};
     const cuuint64_t strides[3] = {(cuuint64_t)p.q_stride[2] * 2, (cuuint64_t)p.q_stride[1] * 2, (cuuint64_t)p.q_stride[0] * 2};
-    const cuuint32_t bw = (cuuint32_t)(W < NC ? W : NC);
     const cuuint32_t box[4] = {64, bw, (cuuint32_t)NC / bw, 1};
-    if (!make_map(&tm_q, q, 4, dims, strides, box)) return ASL_ERR_CUDA;
-  }
-  {
-    const cuuint64_t dims[3] = {128, (cuuint64_t)p.n_kv_heads, (cuuint64_t)c->sum_tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)p.k_stride[1] * 2, (cuuint64_t)p.k_stride[0] * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)KT};
-    if (!make_map(&tm_k, k, 3, dims, strides, box)) return ASL_ERR_CUDA;
+    if (!make_map(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, 4, dims, strides, box)) return ASL_ERR_CUDA;
+    const cuuint64_t kdims[3] = {128, (cuuint64_t)p.n_kv_heads, (cuuint64_t)c->sum_tokens};
+    const cuuint64_t kstr[2] = {(cuuint64_t)p.k_stride[1] * 2, (cuuint64_t)p.k_stride[0] * 2};
+    const cuuint32_t kbox[3] = {64, 1, (cuuint32_t)KT};
+    if (!make_map(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, 3, kdims, kstr, kbox)) return ASL_ERR_CUDA;
   }
   TcArgs a{};
   a.phases = lse ? tp.d_phases2 : tp.d_phases;
@@ -995,8 +1073,14 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.head_dim));
   // every CTA must be resident at once (pass 2 waits for counters other CTAs advance): one CTA per SM at most
   const int grid = tp.grid;
-  if (p.pool_mode == ASL_POOL_MAX) score_tc_kernel<true><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
-  else                             score_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+  const bool per_q = p.pool_mode == ASL_POOL_MAX;
+  if (fp8) {
+    if (per_q) score_tc_kernel<true, true><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+    else       score_tc_kernel<false, true><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+  } else {
+    if (per_q) score_tc_kernel<true, false><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+    else       score_tc_kernel<false, false><<<grid, THREADS, SMEM_BYTES, st>>>(tm_q, tm_k, a);
+  }
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

@@ -10,7 +10,9 @@ constexpr int ASL_TC_KEY_TILE = 128;
 // (T, t_off, tok_off: the request's past length, score offset and first token, copied here so that
 // one record is all a role needs when it enters the phase)
 // rows: query rows of the chunk that exist (the last chunk of a kv head may be padded up to NC)
-struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, rows; };
+// kscale: factor between the accumulator and q.k (1 for bf16 keys; k_scale[h] / 16 for FP8 keys, whose
+// queries are scaled by 16 before they are split into two E4M3 terms)
+struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, rows; float kscale; int32_t pad[3]; };
 
 struct AslTcPlan {
   bool enabled = false;

@@ -272,15 +272,18 @@ def layer_inputs(wl: Workload, layer: int, seed: int = 0, want_v: bool = True) -
     return out
 
 
-def keys_to_fp8(k_bits: np.ndarray):
+def keys_to_fp8(k_bits: np.ndarray, scale=None):
     """An FP8 (E4M3) copy of a layer's keys, as a quantised K cache would hold them: uint8 codes
-    [n][H_k][d] and one fp32 scale per kv head, chosen so that the head's largest magnitude maps to the
-    format's largest finite value (448).  Rounding to nearest by the library cast; input preparation
-    only -- the keys the path is then asked to score ARE code x scale."""
+    [n][H_k][d] and one fp32 scale per kv head, chosen (unless given) so that the head's largest
+    magnitude maps to the format's largest finite value (448).  Rounding to nearest by the library
+    cast; input preparation only -- the keys the path is then asked to score ARE code x scale."""
     import torch
     k = torch.from_numpy(bf16_bits_to_f32(k_bits))
-    amax = k.abs().amax(dim=(0, 2)).clamp_min(1e-30)
-    scale = (amax / 448.0).to(torch.float32)
+    if scale is None:
+        amax = k.abs().amax(dim=(0, 2)).clamp_min(1e-30)
+        scale = (amax / 448.0).to(torch.float32)
+    else:
+        scale = torch.as_tensor(np.asarray(scale, dtype=np.float32))
     codes = (k / scale[None, :, None]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
     return codes.numpy().copy(), scale.numpy().copy()
 

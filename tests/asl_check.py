@@ -29,12 +29,22 @@ def bench_launch(device=0):
 
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
-    """uint16 bf16 bit patterns -> bf16 tensor on cuda:0 (bit-preserving)."""
+    """uint16 bf16 bit patterns -> bf16 tensor on cuda:0 (bit-preserving); uint8 FP8 codes -> uint8 tensor."""
+    if bits.dtype == np.uint8:
+        return torch.from_numpy(bits).cuda()
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
 def bits_of(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.uint8:
+        return t.cpu().numpy()
     return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def with_fp8_keys(x):
+    """The layer's inputs with K replaced by its FP8 copy (codes + one scale per kv head)."""
+    codes, scale = I.keys_to_fp8(x["k"])
+    return {**x, "k": codes, "k_scale": scale}
 
 
 def oracle_layer(wl, x):
@@ -43,7 +53,10 @@ def oracle_layer(wl, x):
     Ps, aggs = [], []
     for b in range(wl.batch):
         q = O.widen_bf16(x["q_obs"][b])
-        k = O.widen_bf16(x["k"][cu[b]:cu[b + 1]])
+        if "k_scale" in x:                       # a quantised K cache: the keys are code x scale
+            k = O.dequantised_keys(x["k"][cu[b]:cu[b + 1]], x["k_scale"])
+        else:
+            k = O.widen_bf16(x["k"][cu[b]:cu[b + 1]])
         P, agg = O.score_layer(q, k, wl.group, wl.pool_kernel, wl.pool_mode)
         Ps.append(P)
         aggs.append(agg)

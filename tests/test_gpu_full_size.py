@@ -76,6 +76,18 @@ def test_million_token_context():
     sweep(wl, 4, range(0, 1))
 
 
+def test_c3_long_context_with_an_fp8_key_cache():
+    """The 128K-token workload with K as FP8 (E4M3) codes, in bench.py's launch configuration."""
+    from paper_2601_07667_b200 import binding as B
+    from asl_check import with_fp8_keys
+    wl = I.workload("C3")
+    x = with_fp8_keys(I.layer_inputs(wl, 0, 0))
+    path = make_path(wl, k_dtype=B.ASL_K_FP8_E4M3, k_scale=[float(s) for s in x["k_scale"]], **bench_launch())
+    check_layer(path, wl, x, 0)
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
 def _benched_launch_case(wl, seed, n_layers):
     """Layers 0..n_layers-1 in bench.py's launch configuration: call by call, then the same layers
     recorded one per CUDA graph and replayed twice over, every output checked against the oracle

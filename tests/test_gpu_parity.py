@@ -9,7 +9,7 @@ import torch
 from oracle import asl_oracle as O
 from paper_2601_07667_b200 import inputs as I
 
-from asl_check import StatReplay, bits_of, check_layer, make_path, to_dev
+from asl_check import StatReplay, bits_of, check_layer, make_path, to_dev, with_fp8_keys
 
 pytestmark = pytest.mark.gpu
 
@@ -147,6 +147,51 @@ def test_a_wait_that_cannot_end_surfaces_as_a_timeout_status(which, code):
     with pytest.raises(B.AslError):
         B.asl_selftest_bounded_wait(path.ctx, 0, 10**9)                 # limits beyond 1 ms are refused
     path.close()
+
+
+@pytest.mark.parametrize("Hq,Hk,w,mode,n", [
+    (32, 8, 64, 0, 128 * 21 + 50),    # 256-row chunks, average pooling
+    (8, 2, 32, 0, 3000),              # 128-row chunk
+    (16, 2, 64, 1, 2100),             # max pooling, two chunks per kv head
+    (28, 4, 64, 0, 1700),             # padded last chunk
+])
+def test_fp8_key_cache(Hq, Hk, w, mode, n):
+    """K as FP8 (E4M3) codes with one scale per kv head: scores against the oracle on the dequantised
+    keys (same tolerance), selection exact on the GPU's scores, K rows compacted as codes, V as bf16."""
+    from paper_2601_07667_b200 import binding as B
+    wl = I.workload("C3", n_q_heads=Hq, n_kv_heads=Hk, window=w, pool_mode=mode, seqlens=(n, n // 2 + 77),
+                    budgets=(w + 200, w + 90), layers=2, l_min=1, l_obs=2)
+    xs = [with_fp8_keys(I.layer_inputs(wl, l, 9)) for l in range(2)]
+    d = wl.head_dim
+    path = None
+    for layer, x in enumerate(xs):
+        if path is None or not np.array_equal(scale, x["k_scale"]):      # the scales belong to the plan
+            if path is not None:
+                path.close()
+            scale = x["k_scale"]
+            path = make_path(wl, k_dtype=B.ASL_K_FP8_E4M3, k_scale=[float(s) for s in scale])
+        check_layer(path, wl, x, layer, check_stat=False)
+        assert path.k_out.dtype == torch.uint8
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
+def test_fp8_keys_are_refused_where_no_tensor_core_path_exists():
+    from paper_2601_07667_b200 import binding as B
+    ctx = B.asl_create(0)
+    base = dict(n_q_heads=8, n_kv_heads=2, head_dim=128, window=24, pool_kernel=7, pool_mode=0,
+                cu_seqlens=[0, 500], budgets=[64], l_min=1, l_obs=2, tau=0.3,
+                q_stride=(8 * 24 * 128, 24 * 128, 128), k_stride=(256, 128), v_stride=(256, 128))
+    with pytest.raises(B.AslError) as e:
+        B.asl_plan(ctx, **base, k_dtype=B.ASL_K_FP8_E4M3, k_scale=[1.0, 1.0])       # W = 24: CUDA-core scorer only
+    assert e.value.status == B.ASL_ERR_UNSUPPORTED
+    ok = {**base, "window": 32, "q_stride": (8 * 32 * 128, 32 * 128, 128)}
+    for bad in (dict(k_scale=None), dict(k_scale=[1.0, 0.0]), dict(k_scale=[1.0, float("inf")]), dict(k_stride=(264, 128))):
+        with pytest.raises(B.AslError) as e:
+            B.asl_plan(ctx, **{**ok, "k_dtype": B.ASL_K_FP8_E4M3, "k_scale": [1.0, 1.0], **bad})
+        assert e.value.status == B.ASL_ERR_INVALID
+    assert B.asl_plan(ctx, **ok, k_dtype=B.ASL_K_FP8_E4M3, k_scale=[0.5, 2.0]) > 0
+    B.asl_destroy(ctx)
 
 
 def test_logits_far_above_the_first_keys_of_a_row():

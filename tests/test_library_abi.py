@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_the_header(lib):
     assert ctypes.sizeof(lib.AslStat) == 64
-    assert ctypes.sizeof(lib.AslParams) == 4 * 10 + 8 + 8 * 2 + 8 * 7
+    assert ctypes.sizeof(lib.AslParams) == 4 * 10 + 8 + 8 * 2 + 8 * 7 + 4 * 2 + 8      # ..., k_dtype, reserved0, k_scale
 
 
 def test_strerror_and_null_handling(lib):
