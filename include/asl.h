@@ -208,13 +208,14 @@ asl_status asl_select_topk(asl_ctx* ctx, const float* scores, int32_t n_heads, i
  * A request is finished at layer l when its record selected at a layer before l.  asl_set_layer tells
  * the context which layer the calls that follow belong to (call it at the start of every layer); the
  * records consulted are those passed to the latest asl_rank_stat call.  Then, for a finished request,
- *   - the scorer leaves out its phases (the flags are read once, ahead of the launch, so a record that a
+ *   - the scorer leaves out its phases (a one-block kernel ahead of the launch reads the flags once and
+ *     writes the launch's phase list without them, so a record that a
  *     still-running asl_rank_stat of the previous layer is about to set takes effect one layer later);
  *   - asl_pool_scores, asl_select_topk and asl_compact_kv leave its scores, kept list and compacted
  *     cache as its selection layer wrote them; they read the records on the device, so issue them after
  *     (on the same stream as, or ordered behind) the asl_rank_stat call of the previous layer;
  *   - its rows of the rank ring are dead: nothing reads or writes them again, the caller may reuse them.
- * Batches of more than 256 requests are scored in full (the other calls still skip).  Without
+ * Batches of more than 4096 requests are scored in full (the other calls still skip).  Without
  * asl_set_layer (or in ASL_CONTROLLER_REPORT) nothing is skipped. */
 enum { ASL_CONTROLLER_REPORT = 0, ASL_CONTROLLER_LATCH = 1 };
 asl_status asl_set_controller(asl_ctx* ctx, int32_t mode);

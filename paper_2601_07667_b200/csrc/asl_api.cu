@@ -13,10 +13,8 @@ void free_plan(asl_ctx* c) {
   asl_tc_free(c);
   if (c->d_req) cudaFree(c->d_req);
   if (c->d_acc) cudaFree(c->d_acc);
-  if (c->d_skip) cudaFree(c->d_skip);
   c->d_req = nullptr;
   c->d_acc = nullptr;
-  c->d_skip = nullptr;
   c->latch_stat = nullptr;
   c->cur_layer = -1;
   c->planned = false;
@@ -118,8 +116,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   if (e == cudaSuccess) e = cudaMemcpy(c->d_req, req.data(), sizeof(AslReq) * p->batch, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&c->d_acc, sizeof(unsigned long long) * (2 * p->batch + 1));
   if (e == cudaSuccess) e = cudaMemset(c->d_acc, 0, sizeof(unsigned long long) * (2 * p->batch + 1));
-  if (e == cudaSuccess) e = cudaMalloc(&c->d_skip, sizeof(uint32_t) * (ASL_SKIP_MAX_BATCH / 32));
-  if (e == cudaSuccess) e = cudaMemset(c->d_skip, 0, sizeof(uint32_t) * (ASL_SKIP_MAX_BATCH / 32));
+
   cudaSetDevice(prev);
   if (e != cudaSuccess) { free_plan(c); return ASL_ERR_CUDA; }
 
@@ -193,10 +190,11 @@ static asl_status score_columns_impl(asl_ctx* c, const void* q_obs, const void* 
   char* ws = static_cast<char*>(workspace);
   float* u = reinterpret_cast<float*>(ws + c->ws.score_u[slot]);
   if (c->tc.enabled) {
-    // requests that have finished are not scored any more: their flags are read once, ahead of the launch,
-    // so that every CTA of the persistent kernel leaves out the same phases
+    // requests that have finished are not scored any more: a small kernel ahead of the launch reads their
+    // flags once and writes the launch's phase list without their phases, so that every CTA of the
+    // persistent kernel walks the same list
     if (c->latch_stat && c->cur_layer >= 0 && c->p.batch <= ASL_SKIP_MAX_BATCH) {
-      const asl_status s = asl_launch_skip_snapshot(c, static_cast<cudaStream_t>(stream));
+      const asl_status s = asl_launch_live_phases(c, lse == nullptr, static_cast<cudaStream_t>(stream));
       if (s != ASL_OK) return s;
     }
     return asl_launch_score_tc(c, q_obs, k, lse, u, ws, static_cast<cudaStream_t>(stream));

@@ -43,7 +43,6 @@ struct asl_ctx {
   int controller = 0;                 // ASL_CONTROLLER_*: asl_set_controller
   const asl_stat* latch_stat = nullptr;   // under ASL_CONTROLLER_LATCH: the records of the latest asl_rank_stat call (device)
   int32_t cur_layer = -1;             // layer the next calls belong to (asl_set_layer / asl_rank_stat)
-  uint32_t* d_skip = nullptr;         // device [8]: bit b set = request b finished before cur_layer (scorer's snapshot)
   asl_params p{};
   std::vector<int32_t> cu, budgets;
   std::vector<float> k_scale;         // per kv head (fp8 K), else empty
@@ -78,7 +77,7 @@ __device__ inline bool asl_finished(const asl_stat* s, int32_t cur) {
   return v->layer_idx < cur;
 }
 #endif
-constexpr int ASL_SKIP_MAX_BATCH = 256;   // requests the scorer's skip mask covers (larger batches are scored in full)
+constexpr int ASL_SKIP_MAX_BATCH = 4096;  // requests the scorer's per-launch phase list covers (larger batches are scored in full)
 
 #define ASL_CUDA(expr)                          \
   do {                                          \
@@ -100,7 +99,7 @@ asl_status asl_launch_wait_selftest(asl_ctx* c, int which, unsigned long long li
 asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const float* lse, float* u, char* ws,
                                cudaStream_t st);
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st);
-asl_status asl_launch_skip_snapshot(asl_ctx* c, cudaStream_t st);
+asl_status asl_launch_live_phases(asl_ctx* c, bool two_pass, cudaStream_t st);
 asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int32_t n_rows, int32_t* ring,
                            asl_stat* stat, char* ws, cudaStream_t st);
 asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* gate,

@@ -87,22 +87,7 @@ __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict_
   if (live) scores_agg[rq.t_off + j] = agg;
 }
 
-// bit b of mask[b / 32]: request b has finished before layer `cur` (read by the scorer launched next)
-__global__ void skip_snapshot_kernel(const asl_stat* __restrict__ latch, int cur, int batch, uint32_t* __restrict__ mask) {
-  const int b = threadIdx.x;
-  const bool fin = b < batch && asl_finished(latch + b, cur);
-  const uint32_t word = __ballot_sync(0xffffffffu, fin);
-  if ((b & 31) == 0) mask[b >> 5] = word;
-}
-
 }  // namespace
-
-asl_status asl_launch_skip_snapshot(asl_ctx* c, cudaStream_t st) {
-  skip_snapshot_kernel<<<1, ASL_SKIP_MAX_BATCH, 0, st>>>(c->latch_stat, c->cur_layer, c->p.batch, c->d_skip);
-  c->launches += 1;
-  ASL_CUDA(cudaGetLastError());
-  return ASL_OK;
-}
 
 asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* scores_agg, cudaStream_t st) {
   const asl_params& p = c->p;

@@ -327,10 +327,11 @@ struct TcArgs {
   uint32_t* folded;        // [segment] rows whose offset is written, accumulated over launches
   int32_t* err;
   int64_t sum_T;
-  const uint32_t* skip_mask;   // null, or bit b set: request b has finished (device-side controller): its phases are left out
   uint32_t* epoch_word;    // two-pass launches completed so far (the counters accumulate over launches); then a ticket word
   uint32_t epoch_limit;    // beyond it the last CTA clears the counters instead of letting them wrap
   int32_t nseg;
+  const int32_t* live_hdr; // null, or device {phases, work items} of `phases`, written ahead of the launch (the list without
+                           // the phases of finished requests); then n_phases / total_items below are not used
   int32_t n_phases, total_items, NC, W, G, Hk, Hq, u_rows_per_kv, u_parts;
   float scale_log2;
 };
@@ -343,8 +344,8 @@ struct ItemWalk {
   int total, n_phases;
   int g, ph;
   TcPhase cur, nxt;
-  __device__ __forceinline__ ItemWalk(const TcArgs& a) : phases(a.phases), total(a.total_items), n_phases(a.n_phases),
-                                                       g((int)blockIdx.x), ph(0) {
+  __device__ __forceinline__ ItemWalk(const TcArgs& a, int n_phases_, int total_) : phases(a.phases), total(total_), n_phases(n_phases_),
+                                                                                g((int)blockIdx.x), ph(0) {
     cur = phases[0];
     nxt = phases[n_phases > 1 ? 1 : 0];
   }
@@ -377,9 +378,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM_MISC + 4);
   volatile uint32_t* s_epoch = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC + 8);
-  volatile uint32_t* s_skip = reinterpret_cast<volatile uint32_t*>(smem + SM_MISC + 16);   // [8]: the launch's copy of the skip mask
-  // every role leaves out the same phases: the item numbering below counts live items only
-  auto skipped = [&](int b) { return b < ASL_SKIP_MAX_BATCH && ((s_skip[b >> 5] >> (b & 31)) & 1u) != 0u; };
+  volatile int* s_list = reinterpret_cast<volatile int*>(smem + SM_MISC + 16);       // {phases, work items} of this launch
+
   float* s_negoff = reinterpret_cast<float*>(smem + SM_NEGOFF);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = a.NC;
@@ -388,8 +388,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // ---- set-up: zero the Q buffers (rows past NC feed unused MMA rows), barriers, tensor memory ----
   if (NC & 127)
     for (int i = threadIdx.x; i < 2 * Q_BUF_BYTES / 16; i += THREADS) reinterpret_cast<uint4*>(smem + SM_Q)[i] = make_uint4(0, 0, 0, 0);
-  if (threadIdx.x >= 32 && threadIdx.x < 32 + ASL_SKIP_MAX_BATCH / 32)
-    s_skip[threadIdx.x - 32] = a.skip_mask ? __ldcg(a.skip_mask + (threadIdx.x - 32)) : 0u;
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(BAR_FULL + s), 1); mbar_init(bar(BAR_EMPTY + s), 1); }
     for (int i = 0; i < 2; ++i) {
@@ -404,6 +402,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint32_t done = 0;
     if (!a.lse) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(done) : "l"(a.epoch_word) : "memory");
     *s_epoch = done + 1u;
+    s_list[0] = a.live_hdr ? __ldcg(a.live_hdr) : a.n_phases;
+    s_list[1] = a.live_hdr ? __ldcg(a.live_hdr + 1) : a.total_items;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -416,12 +416,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
   const uint32_t epoch = *s_epoch;
+  const int n_phases = s_list[0], total_items = s_list[1];
 
   if (warp == 0) {
     // =============================== TMA producer ===============================
     // Local phase l (the l-th phase in which this CTA has a tile) uses Q buffer l%2.
     if (lane == 0) {
-      ItemWalk w(a);
+      ItemWalk w(a, n_phases, total_items);
       const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
       int item = 0, lp = -1, cur_ph = -1;
       int q_issued = -1;                       // highest local phase whose Q chunk has been requested
@@ -456,23 +457,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         q_issued = l;
         return true;
       };
-      for (; ok && w.valid(); w.next()) {
+      for (; ok && w.valid(); w.next(), ++item) {
         const TcPhase p = w.phase();
-        if (skipped(p.b)) continue;
         if (w.ph != cur_ph) {
           cur_ph = w.ph;
           ++lp;
           tok_off = p.tok_off;
           if (q_issued < lp && !issue_q(lp, p, true)) { ok = false; break; }
-          // where does this CTA go after this phase?  (the next phase in which it has a tile and that is not left out)
-          const int grid = (int)gridDim.x;
-          int gn = w.g + ((p.g0 + p.ntiles - w.g + grid - 1) / grid) * grid;
-          int q = w.ph + 1;
+          // where does this CTA go after this phase?
+          const int end = p.g0 + p.ntiles;
+          const int gn = w.g + ((end - w.g + (int)gridDim.x - 1) / (int)gridDim.x) * (int)gridDim.x;
           next_ph = -1;
-          while (gn < a.total_items) {
+          if (gn < w.total) {
+            int q = w.ph + 1;
             while (gn >= a.phases[q].g0 + a.phases[q].ntiles) ++q;
-            if (!skipped(a.phases[q].b)) { next_ph = q; break; }
-            gn += ((a.phases[q].g0 + a.phases[q].ntiles - gn + grid - 1) / grid) * grid;
+            next_ph = q;
           }
         }
         if (next_ph >= 0 && q_issued == lp) {    // prefetch the next phase's Q chunk once its buffer is free
@@ -486,7 +485,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint64_t pol = p.pass == 1 ? pol_keep : pol_stream;
         tma_load_3d(dst, &tm_k, bar(BAR_FULL + s), 0, p.h, tok, pol);
         if (!FP8) tma_load_3d(dst + HALF_BYTES, &tm_k, bar(BAR_FULL + s), 64, p.h, tok, pol);
-        ++item;
       }
       if (!ok) {
         // let the copies already issued land before the CTA's shared memory is released
@@ -502,7 +500,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   } else if (warp == 1) {
     // =============================== MMA issuer =================================
     if (lane == 0) {
-      ItemWalk w(a);
+      ItemWalk w(a, n_phases, total_items);
       int item = 0, lp = -1, cur_ph = -1;
       bool ok = true;
       const uint32_t idesc1 = FP8 ? instr_desc_f8(128, KT) : instr_desc(128, KT);
@@ -511,9 +509,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       auto k_off = [](int ks) { return (uint32_t)(FP8 ? (ks & 3) * 32 : (ks >> 2) * HALF_BYTES + (ks & 3) * 32); };
       const int nhalf = (NC > 128) ? 2 : 1;
       uint32_t qbase = 0;
-      for (; ok && w.valid(); w.next()) {
+      for (; ok && w.valid(); w.next(), ++item) {
         const TcPhase p = w.phase();
-        if (skipped(p.b)) continue;
         if (w.ph != cur_ph) {
           cur_ph = w.ph;
           ++lp;
@@ -548,7 +545,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_commit(bar(BAR_EMPTY + s));       // smem stage free once these MMAs have read it
         tc_commit(bar(BAR_TFULL + acc));     // accumulator ready for the epilogue
         if (w.last_in_phase()) tc_commit(bar(BAR_QEMPTY + (lp & 1)));   // last tile of the phase here
-        ++item;
       }
       if (!ok) {  // make sure nothing is still writing tensor memory before it is freed
         tc_commit(bar(BAR_DRAIN));
@@ -563,9 +559,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int hw = warp - 2;
     const int grid = (int)gridDim.x;
     const int entries = 2 * grid;                                  // entry e: CTA e/2, set e%2
-    for (int ph = 0; ph < a.n_phases; ++ph) {
+    for (int ph = 0; ph < n_phases; ++ph) {
       const TcPhase p = a.phases[ph];
-      if (p.pass != 1 || skipped(p.b)) continue;
+      if (p.pass != 1) continue;
       if ((int)blockIdx.x + hw * grid >= NC) continue;             // no row of this segment is ours
       if (!word_wait(a.published + p.seg, epoch * 2u * (uint32_t)p.ncontrib, s_abort, 41, lane, 256)) break;
       const int first = p.g0 % grid;
@@ -622,7 +618,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     f32x2 scale2 = pk(scale, scale);
     float* negoff = s_negoff + set * 256;
     const int nhalf = (NC > 128) ? 2 : 1;
-    ItemWalk w(a);
+    ItemWalk w(a, n_phases, total_items);
     int item = 0, cur_ph = -1, mine = 0;    // `mine`: tiles this set has taken
     bool dead = false;                      // a wait expired: keep the barrier sequence, skip the work
     // pass-1 state of row sub*128 + lt: sum of 2^(x - mref) over the keys seen so far.  mref is the
@@ -630,9 +626,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // exceed 1, fp32 has the range), unless a sum overflows, in which case the tile is redone with it.
     float mref = -INFINITY, l = 0.f;
     bool first_tile = true;                 // this set has not yet taken a tile of the current pass-1 phase
-    for (; w.valid(); w.next()) {
+    for (; w.valid(); w.next(), ++item) {
       const TcPhase p = w.phase();
-      if (skipped(p.b)) continue;
       if (w.ph != cur_ph) {
         cur_ph = w.ph;
         if (FP8) {
@@ -790,7 +785,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           atomicAdd(a.published + p.seg, 1u);
         }
       }
-      ++item;
     }
   }
 
@@ -811,12 +805,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < 2 * a.nseg; ++i) a.published[i] = 0;      // published and folded are contiguous
         a.epoch_word[0] = 0;
       } else {
-        // segments that were left out: their counters advance as if they had been scored, so that a later
-        // launch that scores them again (a new prompt) finds them where its launch number expects them
-        for (int ph = 0; ph < a.n_phases; ++ph) {
-          const TcPhase q = a.phases[ph];
-          if (q.pass == 1 && skipped(q.b)) { a.published[q.seg] += 2u * (uint32_t)q.ncontrib; a.folded[q.seg] += (uint32_t)NC; }
-        }
         a.epoch_word[0] = epoch;
       }
       __threadfence();
@@ -843,6 +831,56 @@ __global__ void bounded_wait_selftest_kernel(int which, unsigned long long limit
   else            ok = word_wait(never_written, 0xFFFFFFFFu, abort_flag, 92, lane, 256, limit_ns);
   __syncthreads();
   if (threadIdx.x == 0 && !ok && *abort_flag) atomicCAS(err, 0, *abort_flag);
+}
+
+// Device-side controller: the phase list of the next launch without the phases of finished requests.
+// One block.  The requests' flags are read once (a record may be changing under a statistic kernel of the
+// previous layer that is still running: whatever is read here holds for the whole launch), the live
+// phases are copied in order with their first work item recomputed, and the header {phases, items} is
+// written.  Segments that are left out of a two-pass launch have their publish counters advanced as if
+// they had been scored, so that a later launch that scores them again (a new prompt) finds them where
+// its launch number expects them.
+__global__ void __launch_bounds__(256) live_phase_list_kernel(const TcPhase* __restrict__ all, int n_all, const asl_stat* __restrict__ latch,
+                                                             int cur, int batch, int two_pass, int NC, TcPhase* __restrict__ live,
+                                                             int32_t* __restrict__ hdr, uint32_t* __restrict__ published,
+                                                             uint32_t* __restrict__ folded) {
+  __shared__ uint32_t fin[ASL_SKIP_MAX_BATCH / 32];
+  __shared__ int w_items[8], w_cnt[8];
+  __shared__ int base_items, base_cnt;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  for (int b0 = 0; b0 < batch; b0 += 256) {
+    const int b = b0 + tid;
+    const uint32_t word = __ballot_sync(0xffffffffu, b < batch && asl_finished(latch + b, cur));
+    if (lane == 0) fin[b >> 5] = word;
+  }
+  if (tid == 0) { base_items = 0; base_cnt = 0; }
+  __syncthreads();
+  for (int i0 = 0; i0 < n_all; i0 += 256) {
+    const int i = i0 + tid;
+    TcPhase ph{};
+    bool is_live = false;
+    if (i < n_all) {
+      ph = all[i];
+      is_live = ((fin[ph.b >> 5] >> (ph.b & 31)) & 1u) == 0u;
+      if (!is_live && two_pass && ph.pass == 1) { published[ph.seg] += 2u * (uint32_t)ph.ncontrib; folded[ph.seg] += (uint32_t)NC; }
+    }
+    int items = is_live ? ph.ntiles : 0, cnt = is_live ? 1 : 0;
+    int inc_items = items, inc_cnt = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, inc_items, o), c2 = __shfl_up_sync(0xffffffffu, inc_cnt, o);
+      if (lane >= o) { inc_items += a; inc_cnt += c2; }
+    }
+    if (lane == 31) { w_items[wid] = inc_items; w_cnt[wid] = inc_cnt; }
+    __syncthreads();
+    int off_items = base_items + inc_items - items, off_cnt = base_cnt + inc_cnt - cnt;
+    for (int w2 = 0; w2 < wid; ++w2) { off_items += w_items[w2]; off_cnt += w_cnt[w2]; }
+    if (is_live) { ph.g0 = off_items; live[off_cnt] = ph; }
+    __syncthreads();
+    if (tid == 255) { base_items = off_items + items; base_cnt = off_cnt + cnt; }
+    __syncthreads();
+  }
+  if (tid == 0) { hdr[0] = base_cnt; hdr[1] = base_items; }
 }
 
 // FP8 keys: the bf16 window queries, scaled by Q8_SCALE, as two E4M3 terms hi + lo (hi = nearest code,
@@ -974,6 +1012,8 @@ bool asl_tc_plan(asl_ctx* c) {
   if (e == cudaSuccess) e = cudaMalloc(&tp.d_phases2, only2.size() * sizeof(TcPhase));
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases2, only2.data(), only2.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&tp.d_sync, sync_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&tp.d_live, tp.phases.size() * sizeof(TcPhase));
+  if (e == cudaSuccess) e = cudaMalloc(&tp.d_live_hdr, 2 * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemcpy(tp.d_phases, tp.phases.data(), tp.phases.size() * sizeof(TcPhase), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(tp.d_sync, 0, sync_bytes);
   if (e != cudaSuccess) { asl_tc_free(c); return false; }
@@ -996,6 +1036,10 @@ void asl_tc_free(asl_ctx* c) {
   if (tp.d_phases) cudaFree(tp.d_phases);
   if (tp.d_phases2) cudaFree(tp.d_phases2);
   if (tp.d_sync) cudaFree(tp.d_sync);
+  if (tp.d_live) cudaFree(tp.d_live);
+  if (tp.d_live_hdr) cudaFree(tp.d_live_hdr);
+  tp.d_live = nullptr;
+  tp.d_live_hdr = nullptr;
   tp.d_phases = nullptr;
   tp.d_phases2 = nullptr;
   tp.d_sync = nullptr;
@@ -1004,6 +1048,17 @@ void asl_tc_free(asl_ctx* c) {
 
 asl_status asl_launch_wait_selftest(asl_ctx* c, int which, unsigned long long limit_ns, cudaStream_t st) {
   bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(which, limit_ns, reinterpret_cast<const uint32_t*>(c->d_err), c->d_err);   // the error word is never all ones
+  c->launches += 1;
+  ASL_CUDA(cudaGetLastError());
+  return ASL_OK;
+}
+
+asl_status asl_launch_live_phases(asl_ctx* c, bool two_pass, cudaStream_t st) {
+  AslTcPlan& tp = c->tc;
+  const TcPhase* all = two_pass ? tp.d_phases : tp.d_phases2;
+  const int n_all = two_pass ? (int)tp.phases.size() : tp.n_phases2;
+  live_phase_list_kernel<<<1, 256, 0, st>>>(all, n_all, c->latch_stat, c->cur_layer, c->p.batch, two_pass ? 1 : 0, tp.NC, tp.d_live,
+                                            tp.d_live_hdr, tp.d_sync, tp.d_sync + tp.nseg);
   c->launches += 1;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;
@@ -1051,7 +1106,9 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
     if (!make_map(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, 3, kdims, kstr, kbox)) return ASL_ERR_CUDA;
   }
   TcArgs a{};
-  a.phases = lse ? tp.d_phases2 : tp.d_phases;
+  const bool live_list = c->latch_stat && c->cur_layer >= 0 && p.batch <= ASL_SKIP_MAX_BATCH;   // written by asl_launch_live_phases just before
+  a.phases = live_list ? tp.d_live : (lse ? tp.d_phases2 : tp.d_phases);
+  a.live_hdr = live_list ? tp.d_live_hdr : nullptr;
   a.lse = lse;
   a.req = c->d_req;
   a.partials = reinterpret_cast<float2*>(ws + c->ws.score_partials);
@@ -1061,7 +1118,6 @@ asl_status asl_launch_score_tc(asl_ctx* c, const void* q, const void* k, const f
   a.folded = tp.d_sync + tp.nseg;
   a.err = c->d_err;
   a.sum_T = c->sum_T;
-  a.skip_mask = (c->latch_stat && c->cur_layer >= 0 && p.batch <= ASL_SKIP_MAX_BATCH) ? c->d_skip : nullptr;
   a.epoch_word = tp.d_sync + 2 * tp.nseg;         // the one-pass launch touches neither the counters nor this
   a.epoch_limit = 0xFFFFFFFFu / (uint32_t)(2 * tp.grid > MAX_NC ? 2 * tp.grid : MAX_NC) - 2u;
   a.nseg = tp.nseg;

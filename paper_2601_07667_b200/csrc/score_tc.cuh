@@ -12,7 +12,7 @@ constexpr int ASL_TC_KEY_TILE = 128;
 // rows: query rows of the chunk that exist (the last chunk of a kv head may be padded up to NC)
 // kscale: factor between the accumulator and q.k (1 for bf16 keys; k_scale[h] / 16 for FP8 keys, whose
 // queries are scaled by 16 before they are split into two E4M3 terms)
-struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, rows; float kscale; int32_t pad[3]; };
+struct TcPhase { int32_t g0, ntiles, pass, seg, b, h, chunk, ncontrib, T, t_off, tok_off, rows; float kscale; };
 
 struct AslTcPlan {
   bool enabled = false;
@@ -28,4 +28,9 @@ struct AslTcPlan {
   int32_t total_items2 = 0;
   TcPhase* d_phases2 = nullptr;
   uint32_t* d_sync = nullptr;   // [nseg] publish counters, [nseg] folded-row counters, launch number, exit ticket
+  // device-side controller: the phase list of the next launch without the finished requests' phases,
+  // written ahead of the launch (capacity: the longer of the two static lists), and its header
+  // {phases, work items}
+  TcPhase* d_live = nullptr;
+  int32_t* d_live_hdr = nullptr;
 };
