@@ -519,7 +519,7 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": "fp8" if fp8 else "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "seqlens": list(wl.seqlens), "window": wl.window,
                        "budgets": list(wl.budgets), "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv", "d": wl.head_dim,
                        "pool": [wl.pool_kernel, "avg" if wl.pool_mode == 0 else "max"], "k_dtype": args.k_dtype,
