@@ -140,6 +140,7 @@ asl_status asl_plan(asl_ctx* c, const asl_params* p, size_t* workspace_bytes) {
   cudaGetDevice(&prev);
   cudaSetDevice(c->device);
   const bool tc = asl_tc_plan(c);
+  asl_topk_plan(c);
   cudaSetDevice(prev);
   if (fp8 && !tc) { free_plan(c); return ASL_ERR_UNSUPPORTED; }     // only the tensor-core scorer reads 8-bit keys
   const int G = p->n_q_heads / p->n_kv_heads;

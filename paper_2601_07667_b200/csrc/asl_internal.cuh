@@ -60,6 +60,7 @@ struct asl_ctx {
                                       // max pooling: G * u_parts, u_parts consecutive rows per query head)
   int32_t u_parts = 1;                // partial rows per query head under max pooling
   AslTcPlan tc;                       // tensor-core scorer plan (enabled when the shape fits)
+  bool topk_one_cta = false;          // the per-head top-k runs as one CTA per segment (asl_topk_plan)
   AslWorkspace ws{};
   int64_t launches = 0;
 };
@@ -104,6 +105,7 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
                            asl_stat* stat, char* ws, cudaStream_t st);
 asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int32_t* idx_out, const asl_stat* gate,
                            int32_t gate_layer, char* ws, cudaStream_t st);
+bool asl_topk_plan(asl_ctx* c);
 size_t asl_topk_scratch_bytes(int64_t segments, int64_t max_T);
 asl_status asl_launch_compact(asl_ctx* c, const void* k, const void* v, const int32_t* idx, void* k_out, void* v_out,
                               cudaStream_t st);

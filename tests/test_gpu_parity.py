@@ -272,6 +272,54 @@ def test_topk_long_segment_of_many_tiles():
     path.close()
 
 
+def _topk_against_the_oracle(wl, scores):
+    from paper_2601_07667_b200 import binding as B
+    path = make_path(wl)
+    assert scores.shape == (wl.n_kv_heads, path.sum_T)
+    path.scores_kv.copy_(torch.from_numpy(scores))
+    path.idx.fill_(-1)
+    B.asl_select_topk(path.ctx, path.scores_kv, wl.n_kv_heads, path.idx, path.workspace, path.ws_bytes)
+    torch.cuda.synchronize()
+    idx = path.idx.cpu().numpy()
+    for b in range(wl.batch):
+        n, w = wl.seqlens[b], wl.window
+        ts, ko, kept = int(path.t_off[b]), int(path.kept_off[b]), wl.kept(b)
+        for h in range(wl.n_kv_heads):
+            ref = O.select_topk(scores[h, ts:ts + n - w].astype(np.float64), kept - w, n, w)
+            assert (idx[h, ko:ko + kept] == ref).all(), (b, h)
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
+def test_topk_of_mid_sized_segments_heavy_tailed_scores():
+    """Segments of 8 K to 256 K scores (one CTA per segment: a sampled bound, one pass, a short list): smooth
+    heavy-tailed scores, rows that start off a 16-byte boundary, the shortest and the longest such segment."""
+    w = 32
+    for seqlens, budgets in (((131008 + w + 3, 40001 + w), (4096, 2000)), ((8192 + w,), (700,)), ((262144 + w,), (6000,))):
+        wl = I.workload("C1", seqlens=seqlens, budgets=budgets)
+        T = sum(n - w for n in seqlens)
+        rng = np.random.default_rng(T)
+        s = np.exp(rng.normal(-9.0, 1.5, size=(wl.n_kv_heads, T))).astype(np.float32)
+        s[:, :4] += 0.5                      # a few sinks far above the rest
+        _topk_against_the_oracle(wl, s)
+
+
+def test_topk_of_mid_sized_segments_when_the_sampled_bound_fails():
+    """The same kernel where its short list cannot be used: (i) three score levels, so that every score reaches
+    any bound and the list overflows; (ii) the large scores sit exactly on the sampled positions, so that the
+    sample overstates them and fewer than k scores reach the bound.  Either way the result is exact."""
+    w = 32
+    wl = I.workload("C1", seqlens=(50000 + w, 9000 + w), budgets=(3000, 500))
+    _topk_against_the_oracle(wl, I.quantised_scores(wl.n_kv_heads, 59000, 3, seed=4))
+    T = 16384
+    wl = I.workload("C1", seqlens=(T + w,), budgets=(1000 + w,))
+    rng = np.random.default_rng(5)
+    s = rng.uniform(0.0, 1e-3, size=(wl.n_kv_heads, T)).astype(np.float32)
+    sampled = (np.arange(4096, dtype=np.int64) * T) // 4096
+    s[:, sampled[::13]] = rng.uniform(1.0, 2.0, size=(wl.n_kv_heads, sampled[::13].size)).astype(np.float32)
+    _topk_against_the_oracle(wl, s)
+
+
 def test_rank_rows_with_ties_and_statistic_on_planted_rank_rows():
     """asl_rank_stat alone: tied scores, and a ring whose statistic has a closed form."""
     from paper_2601_07667_b200 import binding as B
