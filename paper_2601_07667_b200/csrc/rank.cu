@@ -24,6 +24,28 @@ constexpr int WARPS = SORT_THREADS / 32;
 constexpr int PER_WARP = TILE / WARPS;   // consecutive keys of one warp
 constexpr int ROUNDS = PER_WARP / 32;    // walked 32 at a time, all loads issued up front
 
+// Programmatic dependent launch between the kernels of one rank row: each kernel lets its successor's
+// blocks become resident as soon as its own have started, and the successor waits (for the whole
+// predecessor grid, memory included) only where it first touches what the predecessor writes.  Launched
+// without the attribute both instructions do nothing.
+__device__ __forceinline__ void pdl_release_successor() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ uint32_t desc_key(float s) {
   uint32_t u = __float_as_uint(s);
   if (u == 0x80000000u) u = 0;                           // -0 ranks with +0
@@ -68,6 +90,7 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __r
                                                                 const asl_stat* __restrict__ latch, int nblk, int64_t table,
                                                                 int32_t* __restrict__ hist) {
   __shared__ int cnt[256];
+  pdl_release_successor();
   const int b = blockIdx.y, blk = blockIdx.x;
   const int64_t row = ((int64_t)b * nblk + blk) * 256 + threadIdx.x;
 #pragma unroll
@@ -100,6 +123,8 @@ __global__ void __launch_bounds__(1024) rank_scan(int32_t* __restrict__ hist, co
                                                   const asl_stat* __restrict__ latch, int nblk) {
   __shared__ int part_tot[4][256];
   __shared__ int warp_tot[8];
+  pdl_release_successor();
+  pdl_wait_predecessor();
   const int b = blockIdx.x;
   if (latch && latch[b].selected) return;
   const int used = (req[b].T + TILE - 1) / TILE;             // tiles of this request
@@ -165,6 +190,7 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
                                                              const asl_stat* __restrict__ latch, int shift, int nblk) {
   __shared__ int cnt[WARPS][256];
   __shared__ int warp_tot[WARPS];
+  pdl_release_successor();
   const int b = blockIdx.y, blk = blockIdx.x;
   if (latch && latch[b].selected) return;
   const AslReq rq = req[b];
@@ -175,7 +201,11 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t key[ROUNDS];
   int32_t id[ROUNDS];
+  // the scores were complete before the first histogram ran: the first pass loads them while that kernel
+  // finishes; pairs and counts come from the kernel just before
+  if (!FIRST) pdl_wait_predecessor();
   load_tile<FIRST>(agg, keys_in, idx_in, rq, wstart, lane, key, id);
+  if (FIRST) pdl_wait_predecessor();
   int tile_off;
   if (SCAN) {
     const int used = (rq.T + TILE - 1) / TILE;
@@ -268,14 +298,14 @@ int launch_sort(const float* agg, const AslReq* req, const asl_stat* latch, int 
     int32_t* row = pass == 3 ? rank_row : nullptr;
     int32_t* cur = hist + pass * table;
     int32_t* nxt = pass == 3 ? nullptr : hist + (pass + 1) * table;
-    if (!fused_scan) { rank_scan<<<batch, 1024, 0, st>>>(cur, req, latch, nblk); ++launches; }
+    if (!fused_scan) { launch_after(rank_scan, dim3(batch), dim3(1024), st, cur, req, latch, nblk); ++launches; }
     ++launches;
     if (pass == 0) {
-      if (fused_scan) rank_scatter<true, true><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
-      else rank_scatter<true, false><<<grid, SORT_THREADS, 0, st>>>(agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      if (fused_scan) launch_after(rank_scatter<true, true>, grid, dim3(SORT_THREADS), st, agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      else launch_after(rank_scatter<true, false>, grid, dim3(SORT_THREADS), st, agg, nullptr, nullptr, keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
     } else {
-      if (fused_scan) rank_scatter<false, true><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
-      else rank_scatter<false, false><<<grid, SORT_THREADS, 0, st>>>(nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      if (fused_scan) launch_after(rank_scatter<false, true>, grid, dim3(SORT_THREADS), st, nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
+      else launch_after(rank_scatter<false, false>, grid, dim3(SORT_THREADS), st, nullptr, keys[in], idx[in], keys[out], idx[out], row, cur, nxt, req, latch, shift, nblk);
     }
   }
   return launches;
@@ -340,12 +370,28 @@ __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   unsigned long long num = 0;
   int m = 0;
-  if (j < rq.T && !(a.latch && a.stat[b].selected)) {
-    long long s1 = 0, s2 = 0;
-    int mn = 0x7fffffff;
-    for (int r = 0; r < a.n_rows; ++r) {
-      const int slot = (a.first_layer + r) % a.l_obs;
-      const long long v = a.ring[(int64_t)slot * a.sum_T + rq.t_off + j];
+  const bool live = j < rq.T && !(a.latch && a.stat[b].selected);
+  long long s1 = 0, s2 = 0;
+  int mn = 0x7fffffff;
+  // the rows of the earlier layers are read (eight loads in flight) while the sort of this layer's row ends
+  if (live) {
+    for (int r0 = 0; r0 < a.n_rows - 1; r0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int slot = (a.first_layer + r0 + q) % a.l_obs;
+        v[q] = r0 + q < a.n_rows - 1 ? __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j) : -1;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (v[q] >= 0) { mn = min(mn, v[q]); s1 += v[q]; s2 += (long long)v[q] * v[q]; }
+    }
+  }
+  pdl_wait_predecessor();
+  if (live) {
+    {
+      const int slot = (a.first_layer + a.n_rows - 1) % a.l_obs;
+      const long long v = __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j);
       mn = min(mn, (int)v);
       s1 += v;
       s2 += v * v;
@@ -401,7 +447,7 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
   if (evaluate) {
     StatArgs a{ring, c->d_req, c->d_acc, stat, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows, p.batch, layer_idx,
                latch ? 1 : 0, p.tau};
-    rank_stat_accumulate<<<dim3((c->max_T + 255) / 256, p.batch), 256, 0, st>>>(a);
+    launch_after(rank_stat_accumulate, dim3((c->max_T + 255) / 256, p.batch), dim3(256), st, a);
   } else {
     rank_stat_skip<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, latch ? 1 : 0);
   }
