@@ -46,6 +46,7 @@ def scorer_traffic_bytes(workload_name):
     return None
 # default launch configuration of the timed steps (the GPU parity tests build their paths from the same two values)
 DEFAULT_SCORE_CTAS = -16       # persistent scorer: this many CTAs fewer than SMs (0 = one per SM)
+DEFAULT_LSE_SCORE_CTAS = -32   # the same for the one-pass step (supplied log-sum-exp)
 DEFAULT_TAIL_STREAMS = 2       # side streams for the rest of the layer
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -130,9 +131,11 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(mhz), "reasons": sorted(reasons)}
 
 
-def default_launch(sm_count: int) -> dict:
-    """LayerPath keywords of the launch configuration this benchmark times by default."""
-    ctas = DEFAULT_SCORE_CTAS if DEFAULT_SCORE_CTAS > 0 else max(1, sm_count + DEFAULT_SCORE_CTAS)
+def default_launch(sm_count: int, one_pass: bool = False) -> dict:
+    """LayerPath keywords of the launch configuration this benchmark times by default (``one_pass``: of its
+    one-pass step, scoring with a supplied log-sum-exp)."""
+    want = DEFAULT_LSE_SCORE_CTAS if one_pass else DEFAULT_SCORE_CTAS
+    ctas = want if want > 0 else max(1, sm_count + want)
     return {"score_ctas": ctas, "tail_streams": DEFAULT_TAIL_STREAMS}
 
 
@@ -299,8 +302,13 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = make_workload(args)
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
     if args.score_ctas < 0:
-        args.score_ctas = max(1, torch.cuda.get_device_properties(local).multi_processor_count + args.score_ctas)
+        args.score_ctas = max(1, sms + args.score_ctas)
+    if args.lse_score_ctas is None:
+        args.lse_score_ctas = args.score_ctas
+    elif args.lse_score_ctas < 0:
+        args.lse_score_ctas = max(1, sms + args.lse_score_ctas)
     fp8 = args.k_dtype == "fp8"
     work = algorithmic_work(wl, fp8)
     pk = peaks()
@@ -321,11 +329,14 @@ def run_ours(args):
     dev_sets = [{k: as_dev(t) for k, t in hp.items()} for hp in host_pinned]
     torch.cuda.synchronize()
 
-    path = B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
-                       pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
-                       l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=args.score_ctas,
-                       tail_streams=args.tail_streams, k_dtype=B.ASL_K_FP8_E4M3 if fp8 else B.ASL_K_BF16,
-                       k_scale=None if k_scale is None else [float(s) for s in k_scale])
+    def make_path(score_ctas):
+        return B.LayerPath(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim, window=wl.window,
+                           pool_kernel=wl.pool_kernel, pool_mode=wl.pool_mode, seqlens=wl.seqlens, budgets=wl.budgets,
+                           l_min=wl.l_min, l_obs=wl.l_obs, tau=wl.tau, device=local, score_ctas=score_ctas,
+                           tail_streams=args.tail_streams, k_dtype=B.ASL_K_FP8_E4M3 if fp8 else B.ASL_K_BF16,
+                           k_scale=None if k_scale is None else [float(s) for s in k_scale])
+
+    path = make_path(args.score_ctas)
 
     def barrier():
         if world > 1:
@@ -420,21 +431,22 @@ def run_ours(args):
     stage_ms = [float(np.mean([m[j].elapsed_time(m[j + 1]) for m in marks])) for j in range(4)]
 
     # ---- the same step when the caller supplies the window rows' log-sum-exp (one pass over K) ----
+    lp = path if args.lse_score_ctas == args.score_ctas else make_path(args.lse_score_ctas)
     lse_sets = []
     for ds in dev_sets:
-        B.asl_score_layer(path.ctx, ds["q_obs"], ds["k"], path.scores_kv, path.scores_agg, path.workspace, path.ws_bytes)
+        B.asl_score_layer(lp.ctx, ds["q_obs"], ds["k"], lp.scores_kv, lp.scores_agg, lp.workspace, lp.ws_bytes)
         lse = torch.empty((wl.batch, wl.n_q_heads, wl.window), dtype=torch.float32, device="cuda")
-        B.asl_window_lse(path.ctx, path.workspace, path.ws_bytes, lse)
+        B.asl_window_lse(lp.ctx, lp.workspace, lp.ws_bytes, lse)
         lse_sets.append(lse)
-    path.reset()
+    lp.reset()
     for i in range(args.warmup):
-        path.run_layer(dev_sets[i % n_sets]["q_obs"], dev_sets[i % n_sets]["k"], dev_sets[i % n_sets]["v"], i,
+        lp.run_layer(dev_sets[i % n_sets]["q_obs"], dev_sets[i % n_sets]["k"], dev_sets[i % n_sets]["v"], i,
                        lse=lse_sets[i % n_sets])
-    path.join()
+    lp.join()
     barrier()
     lse_graph = None
     if args.graph:
-        lse_graph = path.capture([step_args(args.warmup + i) + (lse_sets[(args.warmup + i) % n_sets],)
+        lse_graph = lp.capture([step_args(args.warmup + i) + (lse_sets[(args.warmup + i) % n_sets],)
                                   for i in range(args.steps)])
         lse_graph.replay()
         barrier()
@@ -445,11 +457,13 @@ def run_ours(args):
     else:
         for i in range(args.steps):
             j = (args.warmup + i) % n_sets
-            path.run_layer(dev_sets[j]["q_obs"], dev_sets[j]["k"], dev_sets[j]["v"], args.warmup + i, lse=lse_sets[j])
-        path.join()
+            lp.run_layer(dev_sets[j]["q_obs"], dev_sets[j]["k"], dev_sets[j]["v"], args.warmup + i, lse=lse_sets[j])
+        lp.join()
     l1.record(stream)
     barrier()
     lse_ms = max_over_ranks(l0.elapsed_time(l1), world) / args.steps
+    if lp is not path:
+        lp.close()
 
     # ---- end to end through the C ABI with host buffers ----
     e2e_steps = max(2, min(args.steps, args.e2e_steps))
@@ -531,7 +545,7 @@ def run_ours(args):
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_tokens_per_s(wl.total_tokens, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "one_pass_lse": {"ms_per_step": lse_ms, "value": aggregate_tokens_per_s(wl.total_tokens, world, lse_ms),
+            "one_pass_lse": {"ms_per_step": lse_ms, "score_ctas": args.lse_score_ctas, "value": aggregate_tokens_per_s(wl.total_tokens, world, lse_ms),
                              "unit": UNIT, "step_frac": max(t_hbm, t_mma) / (lse_ms * 1e-3),
                              "note": "asl_score_layer_lse: the caller supplies the window rows' log-sum-exp"},
             "gpu_launches": int(launches), "clocks": clocks,
@@ -560,6 +574,9 @@ def main():
     ap.add_argument("--score-ctas", type=int, default=DEFAULT_SCORE_CTAS,
                     help="CTAs of the persistent scorer: 0 = one per SM, negative = that many fewer than SMs.  Fewer "
                          "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")
+    ap.add_argument("--lse-score-ctas", type=int, default=DEFAULT_LSE_SCORE_CTAS,
+                    help="the same for the one-pass step (scoring with a supplied log-sum-exp), whose scorer is short "
+                         "enough for the rest of the layer to want more SMs")
     ap.add_argument("--seqlens", type=str, default=None,
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")

@@ -78,6 +78,30 @@ __device__ inline bool asl_finished(const asl_stat* s, int32_t cur) {
   return v->layer_idx < cur;
 }
 #endif
+// Programmatic dependent launch between consecutive kernels of one stream: a kernel lets its successor's
+// blocks become resident as soon as its own have all started, and a kernel launched with launch_after()
+// waits (for the whole grid before it, memory included) where it first touches what that grid may write.
+// What a kernel reads before the wait must have been complete before its predecessor was launched.
+// Launched the plain way both instructions do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_release_successor() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 constexpr int ASL_SKIP_MAX_BATCH = 4096;  // requests the scorer's per-launch phase list covers (larger batches are scored in full)
 
 #define ASL_CUDA(expr)                          \

@@ -24,7 +24,7 @@ constexpr int HB = 8;            // staged rows per round: their loads are all i
 // rows of u that are added on the way into shared memory.  HB units are staged
 // per round with their halo, pooled from there, and added up per kv head and
 // over all heads in a fixed order: no atomics, bit-reproducible.
-__global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
+__global__ void __launch_bounds__(PT + 2 * MAX_HALO) pool_group_kernel(const float* __restrict__ u, const AslReq* __restrict__ req,
                                                         int Hk, int G, int S, int mode, int urows, int parts, int64_t sum_T,
                                                         const asl_stat* __restrict__ latch, int cur_layer,
                                                         float* __restrict__ scores_kv, float* __restrict__ scores_agg) {
@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict_
   if (j0 >= rq.T) return;
   const int r = S / 2;
   const int j = j0 + threadIdx.x;
-  const bool live = j < rq.T;
+  const bool live = threadIdx.x < PT && j < rq.T;      // the last 2 * MAX_HALO threads only load halo columns
   const int lo = max(0, j - r), hi = min(rq.T - 1, j + r);
   const float inv = 1.0f / (float)S;
   const bool avg = mode == ASL_POOL_AVG;
@@ -48,18 +48,19 @@ __global__ void __launch_bounds__(PT) pool_group_kernel(const float* __restrict_
     const int nb = min(HB, units - u0);
     const int tot = nb * nrows;                       // rows u0*nrows .. u0*nrows + tot - 1 of u
     __syncthreads();
-    for (int i = threadIdx.x; i < PT + 2 * r; i += PT) {
+    if (threadIdx.x < PT + 2 * r) {                     // one column of the tile per thread, halo included
+      const int i = threadIdx.x;
       const int t = j0 - r + i;
       const bool inside = t >= 0 && t < rq.T;
       const float* src = u + (int64_t)u0 * nrows * sum_T + rq.t_off + t;
 #pragma unroll
       for (int q = 0; q < HB; ++q) tile[q][i] = 0.f;
-      for (int e0 = 0; e0 < tot; e0 += 8) {
-        float x[8];
+      for (int e0 = 0; e0 < tot; e0 += 16) {            // sixteen loads in flight
+        float x[16];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = (inside && e0 + k < tot) ? __ldcg(src + (int64_t)(e0 + k) * sum_T) : 0.f;
+        for (int k = 0; k < 16; ++k) x[k] = (inside && e0 + k < tot) ? __ldcg(src + (int64_t)(e0 + k) * sum_T) : 0.f;
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int k = 0; k < 16; ++k)
           if (e0 + k < tot) tile[(e0 + k) / nrows][i] += x[k];
       }
     }
@@ -93,7 +94,7 @@ asl_status asl_launch_pool(asl_ctx* c, const float* u, float* scores_kv, float* 
   const asl_params& p = c->p;
   if (p.pool_kernel / 2 > MAX_HALO) return ASL_ERR_UNSUPPORTED;
   dim3 grid((c->max_T + PT - 1) / PT, p.batch);
-  pool_group_kernel<<<grid, PT, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
+  pool_group_kernel<<<grid, PT + 2 * MAX_HALO, 0, st>>>(u, c->d_req, p.n_kv_heads, p.n_q_heads / p.n_kv_heads, p.pool_kernel,
                                           p.pool_mode, c->u_rows_per_kv, c->u_parts, c->sum_T, c->latch_stat, c->cur_layer,
                                           scores_kv, scores_agg);
   c->launches += 1;

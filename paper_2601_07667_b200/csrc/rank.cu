@@ -24,28 +24,6 @@ constexpr int WARPS = SORT_THREADS / 32;
 constexpr int PER_WARP = TILE / WARPS;   // consecutive keys of one warp
 constexpr int ROUNDS = PER_WARP / 32;    // walked 32 at a time, all loads issued up front
 
-// Programmatic dependent launch between the kernels of one rank row: each kernel lets its successor's
-// blocks become resident as soon as its own have started, and the successor waits (for the whole
-// predecessor grid, memory included) only where it first touches what the predecessor writes.  Launched
-// without the attribute both instructions do nothing.
-__device__ __forceinline__ void pdl_release_successor() { asm volatile("griddepcontrol.launch_dependents;"); }
-__device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-template <typename... KArgs, typename... Args>
-cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 __device__ __forceinline__ uint32_t desc_key(float s) {
   uint32_t u = __float_as_uint(s);
   if (u == 0x80000000u) u = 0;                           // -0 ranks with +0
@@ -90,7 +68,7 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __r
                                                                 const asl_stat* __restrict__ latch, int nblk, int64_t table,
                                                                 int32_t* __restrict__ hist) {
   __shared__ int cnt[256];
-  pdl_release_successor();
+  pdl_release_successor();                 // launched the plain way: the scores are complete when it starts
   const int b = blockIdx.y, blk = blockIdx.x;
   const int64_t row = ((int64_t)b * nblk + blk) * 256 + threadIdx.x;
 #pragma unroll

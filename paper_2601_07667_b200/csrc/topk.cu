@@ -153,10 +153,12 @@ __device__ __forceinline__ void tile_histogram(const Segment& s, const uint32_t 
 // stage 0: digit 1 histogram; stage 1 / 2: pick the previous digit, histogram the next
 template <int STAGE>
 __global__ void __launch_bounds__(THREADS) topk_digit_kernel(TopkArgs a) {
+  pdl_release_successor();
   const Segment s = segment_of(a);
   if (!s.open || s.k == 0 || s.tile * TILE >= s.T) return;
   uint32_t key[PER_THREAD];
-  load_keys(s, key);
+  load_keys(s, key);                      // the scores were complete before the first of these kernels started
+  pdl_wait_predecessor();
   if (STAGE == 0) {
     tile_histogram(s, key, 0u, 0u, 21, 2047u, s.hist);
   } else if (STAGE == 1) {
@@ -177,10 +179,12 @@ __global__ void __launch_bounds__(THREADS) topk_digit_kernel(TopkArgs a) {
 // the k-th largest key and the number of keys equal to it that are kept; per-tile counts
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(TopkArgs a) {
   __shared__ int w_gt[THREADS / 32], w_eq[THREADS / 32];
+  pdl_release_successor();
   const Segment s = segment_of(a);
   if (!s.open || s.k == 0 || s.tile * TILE >= s.T) return;
   uint32_t key[PER_THREAD];
   load_keys(s, key);
+  pdl_wait_predecessor();
   const int bin1 = __ldcg(s.state + 0), bin2 = __ldcg(s.state + 2), rem2 = __ldcg(s.state + 3);
   int bin, need;
   pick<4>(s.hist + 2 * BINS, rem2, bin, need);
@@ -214,11 +218,13 @@ __global__ void __launch_bounds__(THREADS) topk_emit_kernel(TopkArgs a) {
   const Segment s = segment_of(a);
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int tiles = max(1, (s.T + TILE - 1) / TILE);
+  pdl_release_successor();
   if (!s.open || s.tile >= tiles) return;
+  uint32_t key[PER_THREAD];
+  if (s.k) load_keys(s, key);
+  pdl_wait_predecessor();
   for (int t = s.tile * THREADS + tid; t < s.kept - s.k; t += tiles * THREADS) s.out[s.k + t] = s.T + t;   // the window
   if (s.k == 0) return;
-  uint32_t key[PER_THREAD];
-  load_keys(s, key);
   const uint32_t thr = (uint32_t)__ldcg(s.state + 4);
   const int need = __ldcg(s.state + 5);
   // larger / equal keys in the tiles before this one
@@ -720,10 +726,10 @@ asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
   ASL_CUDA(cudaMemsetAsync(a.scratch, 0, (size_t)segments * SEG_INTS * sizeof(int32_t), st));
   const dim3 grid(tiles, n_heads, c->p.batch);
   topk_digit_kernel<0><<<grid, THREADS, 0, st>>>(a);
-  topk_digit_kernel<1><<<grid, THREADS, 0, st>>>(a);
-  topk_digit_kernel<2><<<grid, THREADS, 0, st>>>(a);
-  topk_count_kernel<<<grid, THREADS, 0, st>>>(a);
-  topk_emit_kernel<<<grid, THREADS, 0, st>>>(a);
+  launch_after(topk_digit_kernel<1>, grid, dim3(THREADS), st, a);
+  launch_after(topk_digit_kernel<2>, grid, dim3(THREADS), st, a);
+  launch_after(topk_count_kernel, grid, dim3(THREADS), st, a);
+  launch_after(topk_emit_kernel, grid, dim3(THREADS), st, a);
   c->launches += 5;
   ASL_CUDA(cudaGetLastError());
   return ASL_OK;

@@ -21,11 +21,11 @@ def make_path(wl, device=0, **launch):
                              device=device, **launch)
 
 
-def bench_launch(device=0):
-    """The launch configuration bench.py times by default: the persistent scorer on all but 16 SMs,
-    the rest of the layer on two side streams."""
+def bench_launch(device=0, one_pass=False):
+    """The launch configuration bench.py times by default: the persistent scorer on all but 16 SMs (all but
+    32 for its one-pass step), the rest of the layer on two side streams."""
     import bench
-    return bench.default_launch(torch.cuda.get_device_properties(device).multi_processor_count)
+    return bench.default_launch(torch.cuda.get_device_properties(device).multi_processor_count, one_pass)
 
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:

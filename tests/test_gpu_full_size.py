@@ -117,6 +117,27 @@ def test_c3_benched_launch_calls_and_graph_replay():
     _benched_launch_case(I.workload("C3"), 0, 2)
 
 
+def test_c3_one_pass_step_in_its_benched_launch():
+    """The 128K workload scored in one pass from the oracle's log-sum-exp, in the launch configuration
+    bench.py times that step in, side streams included: every output against the oracle."""
+    from paper_2601_07667_b200 import binding as B
+    from asl_check import O
+    wl = I.workload("C3")
+    x = I.layer_inputs(wl, 0, 0)
+    path = make_path(wl, **bench_launch(one_pass=True))
+    lse_ref = O.window_lse(O.widen_bf16(x["q_obs"][0]), O.widen_bf16(x["k"]), wl.group)
+    lse_dev = torch.from_numpy(lse_ref.astype(np.float32)).cuda().reshape(1, wl.n_q_heads, wl.window)
+    q, k, v = to_dev(x["q_obs"]), to_dev(x["k"]), to_dev(x["v"])
+    for _ in range(2):
+        path.run_layer(q, k, v, 0, lse=lse_dev)
+        path.join()
+        torch.cuda.synchronize()
+        verify_layer(path, wl, x, 0, check_stat=False)
+        path.reset()
+    assert B.asl_device_status(path.ctx)[0] == B.ASL_OK
+    path.close()
+
+
 def test_c4_benched_launch_calls_and_graph_replay():
     _benched_launch_case(I.workload("C4", seed=0), 0, 1)
 
