@@ -23,6 +23,8 @@ constexpr int SORT_THREADS = 256;
 constexpr int WARPS = SORT_THREADS / 32;
 constexpr int PER_WARP = TILE / WARPS;   // consecutive keys of one warp
 constexpr int ROUNDS = PER_WARP / 32;    // walked 32 at a time, all loads issued up front
+constexpr int PARTS = SORT_THREADS / 256;  // threads per digit where a thread walks a digit's column of tile counts
+static_assert(SORT_THREADS % 256 == 0 && SORT_THREADS <= 1024 && TILE % SORT_THREADS == 0, "a thread per digit; whole rounds");
 
 __device__ __forceinline__ uint32_t desc_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -70,15 +72,17 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __r
   __shared__ int cnt[256];
   pdl_release_successor();                 // launched the plain way: the scores are complete when it starts
   const int b = blockIdx.y, blk = blockIdx.x;
-  const int64_t row = ((int64_t)b * nblk + blk) * 256 + threadIdx.x;
+  const int64_t row = ((int64_t)b * nblk + blk) * 256 + (threadIdx.x & 255);
+  if (threadIdx.x < 256) {
 #pragma unroll
-  for (int t = 1; t < 4; ++t) hist[t * table + row] = 0;
+    for (int t = 1; t < 4; ++t) hist[t * table + row] = 0;
+  }
   if (latch && latch[b].selected) return;              // the request's selection is final: no more rank rows
   const AslReq rq = req[b];
   const int start = blk * TILE;
   if (start >= rq.T) return;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  cnt[threadIdx.x] = 0;
+  if (threadIdx.x < 256) cnt[threadIdx.x] = 0;
   uint32_t key[ROUNDS];
   int32_t id[ROUNDS];
   load_tile<true>(agg, nullptr, nullptr, rq, start + wid * PER_WARP, lane, key, id);
@@ -91,7 +95,7 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_hist_first(const float* __r
     if (valid && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&cnt[d], __popc(peers));
   }
   __syncthreads();
-  hist[row] = cnt[threadIdx.x];
+  if (threadIdx.x < 256) hist[row] = cnt[threadIdx.x];
 }
 
 // in place: hist[b][blk][digit] -> first output position of (digit, blk), i.e. the
@@ -166,8 +170,11 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
                                                              int32_t* __restrict__ next_counts,
                                                              const AslReq* __restrict__ req,
                                                              const asl_stat* __restrict__ latch, int shift, int nblk) {
+  constexpr int SCAN_BATCH = 64 / PARTS;       // loads of tile counts in flight per thread
   __shared__ int cnt[WARPS][256];
-  __shared__ int warp_tot[WARPS];
+  __shared__ int warp_tot[8];
+  __shared__ int digit_off[256];
+  __shared__ int part_tot[PARTS > 1 ? PARTS : 1][PARTS > 1 ? 256 : 1], part_before[PARTS > 1 ? PARTS : 1][PARTS > 1 ? 256 : 1];
   pdl_release_successor();
   const int b = blockIdx.y, blk = blockIdx.x;
   if (latch && latch[b].selected) return;
@@ -184,17 +191,31 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
   if (!FIRST) pdl_wait_predecessor();
   load_tile<FIRST>(agg, keys_in, idx_in, rq, wstart, lane, key, id);
   if (FIRST) pdl_wait_predecessor();
-  int tile_off;
   if (SCAN) {
+    // PARTS threads per digit, each over a run of the tiles' counts with all of its loads in flight
+    const int d = threadIdx.x & 255, part = threadIdx.x >> 8;
     const int used = (rq.T + TILE - 1) / TILE;
-    const int32_t* col = counts + (int64_t)b * nblk * 256 + threadIdx.x;
+    const int per = (used + PARTS - 1) / PARTS;
+    const int b0 = part * per, b1 = min(used, b0 + per);
+    const int32_t* col = counts + (int64_t)b * nblk * 256 + d;
     int before = 0, total = 0;
-    for (int i0 = 0; i0 < used; i0 += 32) {          // 32 loads in flight per thread
-      int v[32];
+    for (int i0 = b0; i0 < b1; i0 += SCAN_BATCH) {
+      int v[SCAN_BATCH];
 #pragma unroll
-      for (int k = 0; k < 32; ++k) v[k] = (i0 + k < used) ? __ldcg(col + (int64_t)(i0 + k) * 256) : 0;
+      for (int k = 0; k < SCAN_BATCH; ++k) v[k] = (i0 + k < b1) ? __ldcg(col + (int64_t)(i0 + k) * 256) : 0;
 #pragma unroll
-      for (int k = 0; k < 32; ++k) { total += v[k]; if (i0 + k < blk) before += v[k]; }
+      for (int k = 0; k < SCAN_BATCH; ++k) { total += v[k]; if (i0 + k < blk) before += v[k]; }
+    }
+    if (PARTS > 1) {
+      part_tot[part][d] = total;
+      part_before[part][d] = before;
+      __syncthreads();
+      total = 0;
+      before = 0;
+      if (threadIdx.x < 256) {
+#pragma unroll
+        for (int q = 0; q < PARTS; ++q) { total += part_tot[q][d]; before += part_before[q][d]; }
+      }
     }
     int incl = total;                       // exclusive scan of the digit totals over the 256 digits
 #pragma unroll
@@ -202,12 +223,15 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
       const int v = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += v;
     }
-    if (lane == 31) warp_tot[wid] = incl;
+    if (threadIdx.x < 256 && lane == 31) warp_tot[wid] = incl;
     __syncthreads();
-    tile_off = incl - total + before;
-    for (int w2 = 0; w2 < wid; ++w2) tile_off += warp_tot[w2];
+    if (threadIdx.x < 256) {
+      int off = incl - total + before;
+      for (int w2 = 0; w2 < wid; ++w2) off += warp_tot[w2];
+      digit_off[threadIdx.x] = off;
+    }
   } else {
-    tile_off = counts[((int64_t)b * nblk + blk) * 256 + threadIdx.x];
+    if (threadIdx.x < 256) digit_off[threadIdx.x] = counts[((int64_t)b * nblk + blk) * 256 + threadIdx.x];
   }
   for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&cnt[0][0])[i] = 0;
   __syncthreads();
@@ -222,8 +246,8 @@ __global__ void __launch_bounds__(SORT_THREADS) rank_scatter(const float* __rest
     __syncwarp();
   }
   __syncthreads();
-  {  // digit threadIdx.x: bases of the warps, in warp order, after the tile's global offset
-    int run = tile_off;
+  if (threadIdx.x < 256) {  // digit threadIdx.x: bases of the warps, in warp order, after the tile's global offset
+    int run = digit_off[threadIdx.x];
 #pragma unroll
     for (int w2 = 0; w2 < WARPS; ++w2) {
       const int v = cnt[w2][threadIdx.x];
