@@ -41,7 +41,7 @@ struct TopkArgs {
   int32_t* counts;       // [segments][max_tiles][2]
   int32_t* idx_out;
   int64_t sum_T, sum_kept;
-  int32_t n_heads, max_tiles;
+  int32_t n_heads, max_tiles, max_T;
   const asl_stat* gate;  // null, or: only requests whose statistic selected at layer `gate_layer` are worked on
   int32_t gate_layer;
   const asl_stat* latch; // null, or: requests that finished before layer `cur_layer` are left alone
@@ -304,13 +304,16 @@ struct SegSmem {
   int hist[BINS];
   uint32_t cand_key[SEG_CAP];
   int32_t cand_idx[SEG_CAP];
-  uint32_t bm_gt[SEG_MAX_T / 32];
-  uint32_t bm_eq[SEG_MAX_T / 32];
-  uint16_t pre_gt[SEG_MAX_T / 32], pre_eq[SEG_MAX_T / 32];     // kept scores before each bitmap word (short-list emit)
+  // behind this struct, sized for the plan's longest segment (seg_smem_bytes): two bitmaps over the segment
+  // and, per bitmap word, the kept scores before it (short-list emit)
   int warp_a[SEG_WARPS], warp_b[SEG_WARPS];
   int found[2][2];
   int n_cand;
 };
+
+// dynamic shared memory of the kernel for segments of up to max_T scores
+__host__ __device__ inline int seg_words(int max_T) { return ((max_T + 31) / 32 + 3) & ~3; }
+inline size_t seg_smem_bytes(int max_T) { return sizeof(SegSmem) + (size_t)seg_words(max_T) * (2 * sizeof(uint32_t) + 2 * sizeof(uint16_t)); }
 
 // The sample rank whose key is taken as the lower bound: the expected number of sampled scores among
 // the k largest, plus four standard deviations and two.
@@ -463,6 +466,11 @@ __device__ __forceinline__ void seg_full_hist(SegSmem& sm, const SegWalk& w, uin
 __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a) {
   extern __shared__ __align__(16) uint8_t seg_smem_raw[];
   SegSmem& sm = *reinterpret_cast<SegSmem*>(seg_smem_raw);
+  const int cap_words = seg_words(a.max_T);
+  uint32_t* const bm_gt = reinterpret_cast<uint32_t*>(seg_smem_raw + sizeof(SegSmem));
+  uint32_t* const bm_eq = bm_gt + cap_words;
+  uint16_t* const pre_gt = reinterpret_cast<uint16_t*>(bm_eq + cap_words);
+  uint16_t* const pre_eq = pre_gt + cap_words;
   const Segment s = segment_of(a);
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   if (!s.open) return;
@@ -576,14 +584,14 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
 
   // ---- bitmaps over the segment: keys above the k-th, keys equal to it
   const int words = (s.T + 31) >> 5;
-  for (int i = tid; i < words; i += SEG_THREADS) { sm.bm_gt[i] = 0u; sm.bm_eq[i] = 0u; }
+  for (int i = tid; i < words; i += SEG_THREADS) { bm_gt[i] = 0u; bm_eq[i] = 0u; }
   __syncthreads();
   if (listed) {
     for (int i = tid; i < n; i += SEG_THREADS) {
       const uint32_t key = sm.cand_key[i];
       const int e = sm.cand_idx[i];
-      if (key > thr) atomicOr(&sm.bm_gt[e >> 5], 1u << (e & 31));
-      else if (key == thr) atomicOr(&sm.bm_eq[e >> 5], 1u << (e & 31));
+      if (key > thr) atomicOr(&bm_gt[e >> 5], 1u << (e & 31));
+      else if (key == thr) atomicOr(&bm_eq[e >> 5], 1u << (e & 31));
     }
   } else {
     for (int s0 = w.v_begin; s0 < w.v_end; s0 += 32 * SEG_UNROLL) {
@@ -595,8 +603,8 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
         for (int c = 0; c < 4; ++c)
           if ((m[u] >> c) & 1u) {
             const int e = w.first_index(s0 + 32 * u + lane) + c;
-            if (key[u][c] > thr) atomicOr(&sm.bm_gt[e >> 5], 1u << (e & 31));
-            else if (key[u][c] == thr) atomicOr(&sm.bm_eq[e >> 5], 1u << (e & 31));
+            if (key[u][c] > thr) atomicOr(&bm_gt[e >> 5], 1u << (e & 31));
+            else if (key[u][c] == thr) atomicOr(&bm_eq[e >> 5], 1u << (e & 31));
           }
     }
   }
@@ -606,7 +614,7 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
   const int wpt = (words + SEG_THREADS - 1) / SEG_THREADS;
   const int w0 = min(words, tid * wpt), w1 = min(words, w0 + wpt);
   int cg = 0, ce = 0;
-  for (int i = w0; i < w1; ++i) { cg += __popc(sm.bm_gt[i]); ce += __popc(sm.bm_eq[i]); }
+  for (int i = w0; i < w1; ++i) { cg += __popc(bm_gt[i]); ce += __popc(bm_eq[i]); }
   int ig = cg, ie = ce;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -620,10 +628,10 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
     // every listed score finds its own place: kept scores before its word (at most SEG_CAP: 16 bits) plus those
     // before it in its word; the work is spread evenly however the kept tokens cluster
     for (int i = w0; i < w1; ++i) {
-      sm.pre_gt[i] = (uint16_t)gt_before;
-      sm.pre_eq[i] = (uint16_t)eq_before;
-      gt_before += __popc(sm.bm_gt[i]);
-      eq_before += __popc(sm.bm_eq[i]);
+      pre_gt[i] = (uint16_t)gt_before;
+      pre_eq[i] = (uint16_t)eq_before;
+      gt_before += __popc(bm_gt[i]);
+      eq_before += __popc(bm_eq[i]);
     }
     __syncthreads();
     // places first (they read the listed keys), then the kept indices into the keys' storage in output order,
@@ -638,7 +646,7 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
         if (key >= thr) {
           const int e = sm.cand_idx[i], wd = e >> 5;
           const uint32_t below = (1u << (e & 31)) - 1u;
-          const int g = sm.pre_gt[wd] + __popc(sm.bm_gt[wd] & below), q = sm.pre_eq[wd] + __popc(sm.bm_eq[wd] & below);
+          const int g = pre_gt[wd] + __popc(bm_gt[wd] & below), q = pre_eq[wd] + __popc(bm_eq[wd] & below);
           if (key > thr) place[j] = g + min(q, need);
           else if (q < need) place[j] = g + q;
         }
@@ -654,7 +662,7 @@ __global__ void __launch_bounds__(SEG_THREADS, 1) topk_segment_kernel(TopkArgs a
     return;
   }
   for (int i = w0; i < w1; ++i) {
-    const uint32_t g = sm.bm_gt[i], q = sm.bm_eq[i];
+    const uint32_t g = bm_gt[i], q = bm_eq[i];
     uint32_t bits = g | q;
     while (bits) {
       const int bpos = __ffs(bits) - 1;
@@ -690,7 +698,7 @@ bool asl_topk_plan(asl_ctx* c) {
     const int rank = seg_sample_rank(r.T, r.k) < SEG_SAMPLE ? seg_sample_rank(r.T, r.k) : SEG_SAMPLE;
     if (1.2 * (double)r.T * rank / SEG_SAMPLE > (double)SEG_CAP) return false;
   }
-  if (cudaFuncSetAttribute(topk_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SegSmem)) != cudaSuccess) {
+  if (cudaFuncSetAttribute(topk_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)seg_smem_bytes(c->max_T)) != cudaSuccess) {
     cudaGetLastError();
     return false;
   }
@@ -713,12 +721,13 @@ asl_status asl_launch_topk(asl_ctx* c, const float* scores, int32_t n_heads, int
   a.sum_kept = c->sum_kept;
   a.n_heads = n_heads;
   a.max_tiles = tiles;
+  a.max_T = c->max_T;
   a.gate = gate;
   a.gate_layer = gate_layer;
   a.latch = gate ? nullptr : c->latch_stat;      // the gated call has its own rule
   a.cur_layer = c->cur_layer;
   if (c->topk_one_cta) {
-    topk_segment_kernel<<<dim3(1, n_heads, c->p.batch), SEG_THREADS, sizeof(SegSmem), st>>>(a);
+    topk_segment_kernel<<<dim3(1, n_heads, c->p.batch), SEG_THREADS, seg_smem_bytes(c->max_T), st>>>(a);
     c->launches += 1;
     ASL_CUDA(cudaGetLastError());
     return ASL_OK;
