@@ -698,7 +698,7 @@ bool asl_topk_plan(asl_ctx* c) {
     const int rank = seg_sample_rank(r.T, r.k) < SEG_SAMPLE ? seg_sample_rank(r.T, r.k) : SEG_SAMPLE;
     if (1.2 * (double)r.T * rank / SEG_SAMPLE > (double)SEG_CAP) return false;
   }
-  if (cudaFuncSetAttribute(topk_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)seg_smem_bytes(c->max_T)) != cudaSuccess) {
+  if (cudaFuncSetAttribute(topk_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)seg_smem_bytes(SEG_MAX_T)) != cudaSuccess) {
     cudaGetLastError();
     return false;
   }
