@@ -364,43 +364,56 @@ __global__ void rank_stat_skip(unsigned long long* acc, const AslReq* __restrict
   if (b < batch) stat_finalize_one(acc, req, stat, b, layer_idx, n_rows, 0, 0.0, latch);
 }
 
+constexpr int STAT_TOKENS = 4;   // tokens per thread: few, fat blocks (one wave on the SMs a persistent scorer leaves free)
+
 __global__ void __launch_bounds__(256) rank_stat_accumulate(StatArgs a) {
   __shared__ unsigned long long s_num[8];
   __shared__ int s_m[8];
   const int b = blockIdx.y;
   const AslReq rq = a.req[b];
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool open = !(a.latch && a.stat[b].selected);
   unsigned long long num = 0;
   int m = 0;
-  const bool live = j < rq.T && !(a.latch && a.stat[b].selected);
-  long long s1 = 0, s2 = 0;
-  int mn = 0x7fffffff;
-  // the rows of the earlier layers are read (eight loads in flight) while the sort of this layer's row ends
-  if (live) {
-    for (int r0 = 0; r0 < a.n_rows - 1; r0 += 8) {
-      int v[8];
+  int j[STAT_TOKENS];
+  long long s1[STAT_TOKENS], s2[STAT_TOKENS];
+  int mn[STAT_TOKENS];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const int slot = (a.first_layer + r0 + q) % a.l_obs;
-        v[q] = r0 + q < a.n_rows - 1 ? __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j) : -1;
-      }
+  for (int i = 0; i < STAT_TOKENS; ++i) {
+    j[i] = (blockIdx.x * STAT_TOKENS + i) * 256 + threadIdx.x;
+    s1[i] = 0; s2[i] = 0; mn[i] = 0x7fffffff;
+  }
+  // the rows of the earlier layers are read (all of a batch's loads in flight) while the sort of this layer's row ends
+  for (int r0 = 0; r0 < a.n_rows - 1; r0 += 8) {
+    int v[STAT_TOKENS][8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int slot = (a.first_layer + r0 + q) % a.l_obs;
+#pragma unroll
+      for (int i = 0; i < STAT_TOKENS; ++i)
+        v[i][q] = (open && j[i] < rq.T && r0 + q < a.n_rows - 1) ? __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j[i]) : -1;
+    }
+#pragma unroll
+    for (int i = 0; i < STAT_TOKENS; ++i)
 #pragma unroll
       for (int q = 0; q < 8; ++q)
-        if (v[q] >= 0) { mn = min(mn, v[q]); s1 += v[q]; s2 += (long long)v[q] * v[q]; }
-    }
+        if (v[i][q] >= 0) { mn[i] = min(mn[i], v[i][q]); s1[i] += v[i][q]; s2[i] += (long long)v[i][q] * v[i][q]; }
   }
   pdl_wait_predecessor();
-  if (live) {
-    {
-      const int slot = (a.first_layer + a.n_rows - 1) % a.l_obs;
-      const long long v = __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j);
-      mn = min(mn, (int)v);
-      s1 += v;
-      s2 += v * v;
-    }
-    if (mn < rq.k) {
-      m = 1;
-      num = (unsigned long long)((long long)a.n_rows * s2 - s1 * s1);
+  {
+    const int slot = (a.first_layer + a.n_rows - 1) % a.l_obs;
+    int v[STAT_TOKENS];
+#pragma unroll
+    for (int i = 0; i < STAT_TOKENS; ++i) v[i] = (open && j[i] < rq.T) ? __ldcg(a.ring + (int64_t)slot * a.sum_T + rq.t_off + j[i]) : -1;
+#pragma unroll
+    for (int i = 0; i < STAT_TOKENS; ++i) {
+      if (v[i] < 0) continue;
+      mn[i] = min(mn[i], v[i]);
+      s1[i] += v[i];
+      s2[i] += (long long)v[i] * v[i];
+      if (mn[i] < rq.k) {
+        m += 1;
+        num += (unsigned long long)((long long)a.n_rows * s2[i] - s1[i] * s1[i]);
+      }
     }
   }
 #pragma unroll
@@ -449,7 +462,7 @@ asl_status asl_launch_rank(asl_ctx* c, const float* agg, int32_t layer_idx, int3
   if (evaluate) {
     StatArgs a{ring, c->d_req, c->d_acc, stat, c->sum_T, p.l_obs, layer_idx - n_rows + 1, n_rows, p.batch, layer_idx,
                latch ? 1 : 0, p.tau};
-    launch_after(rank_stat_accumulate, dim3((c->max_T + 255) / 256, p.batch), dim3(256), st, a);
+    launch_after(rank_stat_accumulate, dim3((c->max_T + 256 * STAT_TOKENS - 1) / (256 * STAT_TOKENS), p.batch), dim3(256), st, a);
   } else {
     rank_stat_skip<<<(p.batch + 63) / 64, 64, 0, st>>>(c->d_acc, c->d_req, stat, p.batch, layer_idx, n_rows, latch ? 1 : 0);
   }
