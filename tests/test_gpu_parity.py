@@ -76,6 +76,22 @@ def test_edge_shapes(seqlens, budgets, w, S):
     run_stack(wl, seed=3)
 
 
+@pytest.mark.parametrize("seqlens,w,S", [
+    ((152, 156, 2032 + 32, 36), 32, 9),      # segments of 120, 124, 2032 and 4 past tokens (a warp pools 120): widest window of the kernel
+    ((152, 156, 2032 + 32, 36), 32, 1),      # no neighbours at all
+    ((1000 + 24, 484 + 24), 24, 3),          # one partial row per kv head (the CUDA-core scorer's layout)
+    ((3000 + 64, 1200 + 64), 64, 11),        # a window beyond the kernel's reach: the general kernel on the same layout
+    ((3000 + 64, 1201 + 64), 64, 7),         # second segment off a 16-byte boundary: the general kernel
+])
+def test_average_pooling_on_aligned_segments(seqlens, w, S):
+    """Batches whose segments all start and end on 16-byte boundaries of the score rows take the pooling kernel
+    without shared memory; lengths around a warp's 120 tokens, every window size it covers, and the neighbouring
+    cases that fall back to the general kernel."""
+    wl = I.workload("C1", seqlens=seqlens, budgets=tuple(w + max(1, (n - w) // 4) for n in seqlens), window=w, pool_kernel=S,
+                    layers=2, l_min=1, l_obs=2)
+    run_stack(wl, seed=6)
+
+
 @pytest.mark.parametrize("Hq,Hk,w,mode,n", [
     (32, 8, 64, 0, 3000),     # 256-row chunks, average pooling (the 8B-shaped layout)
     (8, 2, 128, 0, 2500),     # two 256-row chunks per kv head, average pooling
