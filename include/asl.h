@@ -119,7 +119,7 @@ typedef struct {
   int32_t reserved;
   double var_top;     /* num / (rows^2 * m)                                               */
   double init_var;    /* var_top at the first evaluated layer                             */
-  double rel;         /* var_top / init_var                                               */
+  double rel;         /* var_top / init_var (NaN, which never selects, if init_var is 0)  */
 } asl_stat;
 
 /* Context bound to CUDA device `device`.  ASL_ERR_ARCH unless it is sm_100. */

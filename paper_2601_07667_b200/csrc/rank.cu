@@ -345,7 +345,7 @@ __device__ void stat_finalize_one(unsigned long long* acc, const AslReq* __restr
     s.evaluated = 1;
     s.var_top = (double)num / ((double)n_rows * (double)n_rows * (double)m);   // empty union (k = 0): NaN, never selects
     if (!s.has_init) { s.init_var = s.var_top; s.has_init = 1; }
-    s.rel = s.var_top / s.init_var;
+    s.rel = s.init_var != 0.0 ? s.var_top / s.init_var : __longlong_as_double(0x7ff8000000000000ll);   // zero first variance: undefined, never selects
     s.selected = (s.rel < tau) ? 1 : 0;
   }
   const int32_t selected = s.selected;

@@ -169,8 +169,8 @@ class StatReplay:
                     assert np.isnan(s["var_top"]) and np.isnan(s["rel"]) and np.isnan(iso["rel"])
                 else:
                     assert abs(s["var_top"] - iso["var_top"]) <= 1e-14 * abs(iso["var_top"])
-                    if np.isnan(iso["rel"]):   # the first evaluated layer had zero variance: the ratio is undefined (0/0 or x/0) and never selects
-                        assert not np.isfinite(s["rel"]) and not bool(s["selected"])
+                    if np.isnan(iso["rel"]):   # the first evaluated layer had zero variance: the ratio is undefined and never selects
+                        assert np.isnan(s["rel"]) and not bool(s["selected"])
                     else:
                         assert abs(s["rel"] - iso["rel"]) <= 1e-13 * abs(iso["rel"])
                 assert bool(s["selected"]) == iso["selected"]
