@@ -257,6 +257,20 @@ def test_controller_policy():
     assert sel[-2] > 3           # the comparison is strict: rel = 1.0 is not < 1.0
 
 
+def test_controller_after_a_first_layer_without_variance():
+    """Rank rows that agree on the union at the first evaluated layer give var_top = 0: every later ratio to
+    it is undefined (NaN) and the strict comparison never fires, whatever the threshold."""
+    T = 40
+    same = np.linspace(1.0, 0.0, T)                      # the same order at every layer: identical rank rows
+    c = O.SelectionController(budget=8 + 4, window=4, l_min=1, l_obs=2, tau=10.0)
+    outs = [c.step(l, same) for l in range(2)]
+    assert outs[1]["evaluated"] and outs[1]["var_top"] == 0.0 and np.isnan(outs[1]["rel"]) and not outs[1]["selected"]
+    moved = same.copy()
+    moved[[0, 30]] = moved[[30, 0]]                      # now the rows differ: the variance is positive, the ratio still undefined
+    out = c.step(2, moved)
+    assert out["var_top"] > 0.0 and np.isnan(out["rel"]) and not out["selected"] and c.selected_layer < 0
+
+
 # ------------------------------------------------------------------ O7 / O8
 def test_select_topk_brute_force_ties_and_edges():
     g = rng(40)
