@@ -47,8 +47,8 @@ def scorer_traffic_bytes(workload_name):
 # default launch configuration of the timed steps (the GPU parity tests build their paths from the same two values)
 DEFAULT_WORKLOAD = "C3"
 DEFAULT_SCORE_CTAS = -16       # persistent scorer: this many CTAs fewer than SMs (0 = one per SM)
-DEFAULT_LSE_SCORE_CTAS = -32   # the same for the one-pass step (supplied log-sum-exp) of the default workload, whose
-                               # scorer is short enough for the rest of the layer to want more SMs; other workloads: as above
+DEFAULT_LSE_SCORE_CTAS = -32   # the same for the one-pass step (supplied log-sum-exp) where a kv head has at most 256 query
+                               # rows: its scorer is short enough for the rest of the layer to want more SMs; else as above
 DEFAULT_TAIL_STREAMS = 2       # side streams for the rest of the layer
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -307,7 +307,7 @@ def run_ours(args):
     sms = torch.cuda.get_device_properties(local).multi_processor_count
     if args.score_ctas < 0:
         args.score_ctas = max(1, sms + args.score_ctas)
-    if args.lse_score_ctas is None and args.workload == DEFAULT_WORKLOAD and args.seqlens is None:
+    if args.lse_score_ctas is None and (wl.n_q_heads // wl.n_kv_heads) * wl.window <= 256:
         args.lse_score_ctas = DEFAULT_LSE_SCORE_CTAS
     if args.lse_score_ctas is None:
         args.lse_score_ctas = args.score_ctas
@@ -580,7 +580,7 @@ def main():
                          "leaves SMs to the previous layer's statistic, top-k and compaction, which run on a side stream")
     ap.add_argument("--lse-score-ctas", type=int, default=None,
                     help="the same for the one-pass step (scoring with a supplied log-sum-exp); default: "
-                         f"{DEFAULT_LSE_SCORE_CTAS} for the default workload, else --score-ctas")
+                         f"{DEFAULT_LSE_SCORE_CTAS} where a kv head has at most 256 query rows, else --score-ctas")
     ap.add_argument("--seqlens", type=str, default=None,
                     help="comma-separated context lengths replacing the workload's (smaller cases for profiling)")
     ap.add_argument("--budgets", type=str, default=None, help="comma-separated KV budgets, one per request")
