@@ -20,12 +20,12 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const uint8_t* __restri
   const int64_t orow = (int64_t)h * sum_kept + rq.kept_off + r;
   const int64_t tok = (int64_t)rq.tok_off + idx[orow];
   if (c < k_vec) {
-    const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * ks_t + (int64_t)h * ks_h + c * 16);
-    *reinterpret_cast<uint4*>(k_out + (orow * k_vec + c) * 16) = kv;
+    const uint4 kv = __ldcs(reinterpret_cast<const uint4*>(k + tok * ks_t + (int64_t)h * ks_h + c * 16));
+    __stcs(reinterpret_cast<uint4*>(k_out + (orow * k_vec + c) * 16), kv);
   }
   if (c < v_vec) {
-    const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * vs_t + (int64_t)h * vs_h + c * 16);
-    *reinterpret_cast<uint4*>(v_out + (orow * v_vec + c) * 16) = vv;
+    const uint4 vv = __ldcs(reinterpret_cast<const uint4*>(v + tok * vs_t + (int64_t)h * vs_h + c * 16));
+    __stcs(reinterpret_cast<uint4*>(v_out + (orow * v_vec + c) * 16), vv);
   }
 }
 
